@@ -1,0 +1,443 @@
+/*
+ * cdq_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, fp64 CPU statement of the CDQuant per-layer pipeline, written
+ * from the paper so that the CUDA library can be checked against it.  Only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg may use it; the
+ * CUDA library shares no code with it and never calls it.
+ *
+ * What it computes (paper, Section 3):
+ *   - H = X^T X                                   (Notation; Algorithm 1 line 2)
+ *   - MinMax / OWC grid and round-to-nearest codes (Eq. 2 and the grid search
+ *     over the clipping strength gamma that follows it; per-group form of the
+ *     "Initialization" paragraph of the sub-channel section)
+ *   - gradient of the layer loss                   (Algorithm 1 line 3)
+ *   - greedy coordinate descent                    (Algorithm 1 lines 4-8;
+ *     Algorithm 4 for sub-channel grids)
+ *   - the layer loss  sum_j e_j^T H e_j            (Eq. 1 written with H)
+ *
+ * Formulation.  Algorithm 1 works in code units (g = 2H(q - (w-b)/a), the
+ * printed decrease (r-q_i)^2 H_ii + (r-q_i) g_i is the loss change divided by
+ * a^2).  Algorithm 4 rescales X by the per-coordinate scales, which gives a
+ * different matrix for every output column.  Both are the same iteration as
+ * the weight-unit form used here,
+ *        G = 2 H (w_hat - w),   d = a_i (r - q_i),
+ *        Delta(i, r) = d^2 H_ii + d G_i      (the true change of the loss),
+ *        G <- G + 2 d H[i*, :]
+ * because g_tilde = D_a G and H_tilde_ii = a_i^2 H_ii.  cdqo_cd_code_units()
+ * below is the literal code-unit iteration of Algorithm 1 / Algorithm 4 and
+ * the tests check that both pick the same moves.
+ *
+ * Fixed readings where the paper is silent:
+ *   - ties: lowest coordinate i, then lowest level r; a move is taken only if
+ *     it strictly lowers the loss (the no-op r = q_i has Delta = 0), otherwise
+ *     the column is finished;
+ *   - rounding in Eq. 2 is round-half-to-even;
+ *   - OWC keeps b = min(w) and shrinks only a (Eq. 2 taken literally); with
+ *     groups, one gamma per output column is applied to every group of it and
+ *     is chosen on the full column loss;
+ *   - scale a and zero b are stored as fp32 (what a dequantiser would hold);
+ *   - H handed from one stage to the next is fp32 (the library's H is fp32).
+ *
+ * Arithmetic: fp64 everywhere, sums in ascending index order, no fused
+ * multiply-add (build with -ffp-contract=off) so that an fp64 device kernel
+ * that follows the same order can match bit for bit.
+ *
+ * Pins (tests/test_oracle_*.py): brute force over all codes on tiny layers;
+ * Delta against the loss recomputed from X; incremental G against a fresh
+ * 2H(w_hat-w); monotone loss; closed-form coordinate optimum against the level
+ * scan; diagonal H => no move; gamma = 1 => MinMax; code-unit Algorithm 4 ==
+ * weight-unit picks; local optimality at convergence; d_in = 1.
+ * Parity unpinned: anything that depends on the paper's (unstated) lambda.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef long long i64;
+
+int cdqo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------ */
+/* H = X^T X  (Notation paragraph of Section 3; Algorithm 1 line 2).         */
+/* X: [n, d_in] row-major, already widened exactly to fp64.                  */
+/* H64: [d_in, d_in] fp64 result; H32 (may be NULL): the same rounded to     */
+/* fp32, which is what every later stage consumes.                           */
+/* lambda_rel > 0 adds lambda_rel * mean(diag H) to the diagonal (the        */
+/* "lambda I" regulariser of Section 4; the paper does not give its value).  */
+/* ------------------------------------------------------------------------ */
+int cdqo_hessian(const double* X, i64 n, i64 d_in, double lambda_rel,
+                 double* H64, float* H32) {
+  if (!X || !H64 || n < 0 || d_in <= 0) return 1;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (i64 p = 0; p < d_in; ++p) {
+    double* row = H64 + p * d_in;
+    for (i64 r = 0; r < d_in; ++r) row[r] = 0.0;
+    for (i64 k = 0; k < n; ++k) {
+      const double xp = X[k * d_in + p];
+      const double* xr = X + k * d_in;
+      for (i64 r = 0; r < d_in; ++r) row[r] = row[r] + xp * xr[r];
+    }
+  }
+  if (lambda_rel > 0.0) {
+    double tr = 0.0;
+    for (i64 p = 0; p < d_in; ++p) tr = tr + H64[p * d_in + p];
+    const double add = lambda_rel * (tr / (double)d_in);
+    for (i64 p = 0; p < d_in; ++p) H64[p * d_in + p] = H64[p * d_in + p] + add;
+  }
+  if (H32)
+    for (i64 e = 0; e < d_in * d_in; ++e) H32[e] = (float)H64[e];
+  return 0;
+}
+
+/* Selected entries of H = X^T X: out[s] = sum_k X[k,rows[s]] X[k,cols[s]].  */
+int cdqo_hessian_entries(const double* X, i64 n, i64 d_in, const i64* rows,
+                         const i64* cols, i64 n_entries, double* out) {
+  if (!X || !rows || !cols || !out) return 1;
+#pragma omp parallel for schedule(static)
+  for (i64 s = 0; s < n_entries; ++s) {
+    double acc = 0.0;
+    for (i64 k = 0; k < n; ++k)
+      acc = acc + X[k * d_in + rows[s]] * X[k * d_in + cols[s]];
+    out[s] = acc;
+  }
+  return 0;
+}
+
+/* gamma_k of the clipping grid: lo + (hi-lo)*k/(n_clip-1); a one-point grid */
+/* is MinMax (gamma = 1).                                                    */
+double cdqo_gamma(int k, int n_clip, double lo, double hi) {
+  if (n_clip <= 1) return 1.0;
+  return lo + ((hi - lo) * (double)k) / (double)(n_clip - 1);
+}
+
+/* Eq. 2 for one group of one column: w[0..len) with stride 1.               */
+static void grid_rtn_group(const double* w, i64 len, int L, double gamma,
+                           float* a_out, float* b_out, uint8_t* q) {
+  double mn = w[0], mx = w[0];
+  for (i64 i = 1; i < len; ++i) {
+    if (w[i] < mn) mn = w[i];
+    if (w[i] > mx) mx = w[i];
+  }
+  const float b32 = (float)mn;
+  const float a32 = (float)((gamma * (mx - mn)) / (double)L);
+  *a_out = a32;
+  *b_out = b32;
+  if (!(a32 > 0.0f)) { /* constant group: every code 0, nothing to move */
+    for (i64 i = 0; i < len; ++i) q[i] = 0;
+    return;
+  }
+  const double a = (double)a32, b = (double)b32;
+  for (i64 i = 0; i < len; ++i) {
+    double r = rint((w[i] - b) / a); /* round half to even */
+    if (r < 0.0) r = 0.0;
+    if (r > (double)L) r = (double)L;
+    q[i] = (uint8_t)r;
+  }
+}
+
+/* e = (a*q + b) - w for one column. */
+static void residual(const double* w, const uint8_t* q, const float* a,
+                     const float* b, i64 d_in, i64 g, double* e) {
+  for (i64 i = 0; i < d_in; ++i) {
+    const double ai = (double)a[i / g], bi = (double)b[i / g];
+    e[i] = (ai * (double)q[i] + bi) - w[i];
+  }
+}
+
+/* e^T H e, sums ascending. he (scratch, d_in) receives H e. */
+static double quad_form(const float* H, const double* e, i64 d_in, double* he) {
+  double loss = 0.0;
+  for (i64 p = 0; p < d_in; ++p) {
+    const float* row = H + p * d_in;
+    double acc = 0.0;
+    for (i64 k = 0; k < d_in; ++k) acc = acc + (double)row[k] * e[k];
+    he[p] = acc;
+  }
+  for (i64 p = 0; p < d_in; ++p) loss = loss + e[p] * he[p];
+  return loss;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Grid + round-to-nearest, with the OWC grid search when n_clip > 1         */
+/* (Eq. 2 and the minimisation over gamma stated right after it).            */
+/* W: [d_in, d_out] row-major fp64 (widened).  group_size 0 => per-channel.  */
+/* scale, zero: [d_in/g, d_out] fp32.  Q: [d_in, d_out] u8.                  */
+/* gamma_idx (may be NULL): [d_out] chosen grid index.                       */
+/* loss_table (may be NULL): [n_clip, d_out] loss of every gamma.            */
+/* H (fp32, [d_in,d_in]) is needed only when n_clip > 1.                     */
+/* ------------------------------------------------------------------------ */
+int cdqo_init_rtn(const double* W, i64 d_in, i64 d_out, const float* H,
+                  int bits, i64 group_size, int n_clip, double clip_lo,
+                  double clip_hi, float* scale, float* zero, uint8_t* Q,
+                  int* gamma_idx, double* loss_table) {
+  if (!W || !scale || !zero || !Q || bits < 1 || bits > 8 || d_in <= 0 || d_out <= 0)
+    return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g) return 2;
+  if (n_clip > 1 && !H) return 1;
+  const i64 ng = d_in / g;
+  const int L = (1 << bits) - 1;
+  const int nk = n_clip > 1 ? n_clip : 1;
+#pragma omp parallel
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    double* he = (double*)malloc(sizeof(double) * d_in);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) w[i] = W[i * d_out + j];
+      int best_k = 0;
+      if (nk > 1) {
+        double best = 0.0;
+        for (int k = 0; k < nk; ++k) {
+          const double gamma = cdqo_gamma(k, nk, clip_lo, clip_hi);
+          for (i64 t = 0; t < ng; ++t)
+            grid_rtn_group(w + t * g, g, L, gamma, a + t, b + t, q + t * g);
+          residual(w, q, a, b, d_in, g, e);
+          const double loss = quad_form(H, e, d_in, he);
+          if (loss_table) loss_table[(i64)k * d_out + j] = loss;
+          if (k == 0 || loss < best) { best = loss; best_k = k; }
+        }
+      }
+      const double gamma = cdqo_gamma(best_k, nk, clip_lo, clip_hi);
+      for (i64 t = 0; t < ng; ++t)
+        grid_rtn_group(w + t * g, g, L, gamma, a + t, b + t, q + t * g);
+      for (i64 t = 0; t < ng; ++t) {
+        scale[t * d_out + j] = a[t];
+        zero[t * d_out + j] = b[t];
+      }
+      for (i64 i = 0; i < d_in; ++i) Q[i * d_out + j] = q[i];
+      if (gamma_idx) gamma_idx[j] = best_k;
+    }
+    free(w); free(e); free(he); free(q); free(a); free(b);
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Gradient G = 2 H (w_hat - w) for every column (Algorithm 1 line 3 in      */
+/* weight units).  G: [d_out, d_in] fp64, one column of the layer per row.   */
+/* ------------------------------------------------------------------------ */
+int cdqo_gradient(const float* H, const double* W, i64 d_in, i64 d_out,
+                  i64 group_size, const float* scale, const float* zero,
+                  const uint8_t* Q, double* G) {
+  if (!H || !W || !scale || !zero || !Q || !G) return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g) return 2;
+  const i64 ng = d_in / g;
+#pragma omp parallel
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) { w[i] = W[i * d_out + j]; q[i] = Q[i * d_out + j]; }
+      for (i64 t = 0; t < ng; ++t) { a[t] = scale[t * d_out + j]; b[t] = zero[t * d_out + j]; }
+      residual(w, q, a, b, d_in, g, e);
+      for (i64 p = 0; p < d_in; ++p) {
+        const float* row = H + p * d_in;
+        double acc = 0.0;
+        for (i64 k = 0; k < d_in; ++k) acc = acc + (double)row[k] * e[k];
+        G[j * d_in + p] = 2.0 * acc;
+      }
+    }
+    free(w); free(e); free(q); free(a); free(b);
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Greedy coordinate descent, weight-unit form (Algorithm 1 lines 4-8; the   */
+/* sub-channel Algorithm 4 is the same iteration, see the header).           */
+/* Q is updated in place.  T = passes * d_in steps per column at most.       */
+/* stats_u64[3] = {steps budget (T*d_out), committed moves, columns that ran */
+/* out of improving moves}; loss_ba[2] = {loss before, loss after}, both     */
+/* recomputed from scratch as sum_j e_j^T H e_j.                             */
+/* trace_* (may be NULL): for column trace_col, the move of every committed  */
+/* step (capacity T): coordinate, new level, Delta.                          */
+/* moves_per_col (may be NULL): [d_out] committed moves of each column.      */
+/* G_final (may be NULL): [d_out, d_in] the incrementally kept gradient.     */
+/* ------------------------------------------------------------------------ */
+int cdqo_cd_solve(const float* H, const double* W, i64 d_in, i64 d_out, int bits,
+                  i64 group_size, const float* scale, const float* zero,
+                  uint8_t* Q, i64 steps_per_col, unsigned long long* stats_u64,
+                  double* loss_ba, i64 trace_col, int* trace_i, int* trace_r,
+                  double* trace_delta, i64* moves_per_col, double* G_final) {
+  if (!H || !W || !scale || !zero || !Q || bits < 1 || bits > 8) return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g) return 2;
+  const i64 ng = d_in / g;
+  const int L = (1 << bits) - 1;
+  const i64 T = steps_per_col;
+  unsigned long long committed = 0, converged = 0;
+  double* lb = (double*)malloc(sizeof(double) * d_out);
+  double* la = (double*)malloc(sizeof(double) * d_out);
+#pragma omp parallel reduction(+ : committed, converged)
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    double* G = (double*)malloc(sizeof(double) * d_in);
+    double* he = (double*)malloc(sizeof(double) * d_in);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) { w[i] = W[i * d_out + j]; q[i] = Q[i * d_out + j]; }
+      for (i64 t = 0; t < ng; ++t) { a[t] = scale[t * d_out + j]; b[t] = zero[t * d_out + j]; }
+      residual(w, q, a, b, d_in, g, e);
+      lb[j] = quad_form(H, e, d_in, he);
+      for (i64 p = 0; p < d_in; ++p) G[p] = 2.0 * he[p];
+      i64 moves = 0;
+      int done = 0;
+      for (i64 t = 0; t < T; ++t) {
+        double best = 0.0; /* the no-op */
+        i64 bi = -1;
+        int br = 0;
+        double bd = 0.0;
+        for (i64 i = 0; i < d_in; ++i) {
+          const double ai = (double)a[i / g];
+          const double hii = (double)H[i * d_in + i];
+          const int qi = (int)q[i];
+          for (int r = 0; r <= L; ++r) {
+            if (r == qi) continue;
+            const double d = ai * (double)(r - qi);
+            const double delta = (d * d) * hii + d * G[i];
+            if (delta < best) { best = delta; bi = i; br = r; bd = d; }
+          }
+        }
+        if (bi < 0) { done = 1; break; }
+        if (j == trace_col && trace_i) {
+          trace_i[moves] = (int)bi; trace_r[moves] = br; trace_delta[moves] = best;
+        }
+        q[bi] = (uint8_t)br;
+        const float* row = H + bi * d_in; /* H symmetric: column i* = row i* */
+        const double two_d = 2.0 * bd;
+        for (i64 p = 0; p < d_in; ++p) G[p] = G[p] + two_d * (double)row[p];
+        ++moves;
+      }
+      committed += (unsigned long long)moves;
+      converged += (unsigned long long)done;
+      if (moves_per_col) moves_per_col[j] = moves;
+      if (G_final) for (i64 p = 0; p < d_in; ++p) G_final[j * d_in + p] = G[p];
+      for (i64 i = 0; i < d_in; ++i) Q[i * d_out + j] = q[i];
+      residual(w, q, a, b, d_in, g, e);
+      la[j] = quad_form(H, e, d_in, he);
+    }
+    free(w); free(e); free(G); free(he); free(q); free(a); free(b);
+  }
+  double loss_before = 0.0, loss_after = 0.0;
+  for (i64 j = 0; j < d_out; ++j) { /* ascending j */
+    loss_before = loss_before + lb[j];
+    loss_after = loss_after + la[j];
+  }
+  free(lb); free(la);
+  if (stats_u64) {
+    stats_u64[0] = (unsigned long long)T * (unsigned long long)d_out;
+    stats_u64[1] = committed;
+    stats_u64[2] = converged;
+  }
+  if (loss_ba) { loss_ba[0] = loss_before; loss_ba[1] = loss_after; }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* The literal code-unit iteration for ONE column: Algorithm 4 (which is     */
+/* Algorithm 1 when the scale is one constant): H_t = D_a H D_a,             */
+/* g = 2 H_t (q0 - (w - b)/a), decrease (r-q_i)^2 H_t,ii + (r-q_i) g_i.      */
+/* Records the committed moves; used only to check the weight-unit form.     */
+/* a_full, b_full: per-coordinate scale and zero, all a_full > 0.            */
+/* Returns the number of moves.                                              */
+/* ------------------------------------------------------------------------ */
+i64 cdqo_cd_code_units(const float* H, const double* w, const double* a_full,
+                       const double* b_full, i64 d_in, int bits, uint8_t* q,
+                       i64 T, int* trace_i, int* trace_r) {
+  const int L = (1 << bits) - 1;
+  double* Ht = (double*)malloc(sizeof(double) * d_in * d_in);
+  double* gt = (double*)malloc(sizeof(double) * d_in);
+  double* z = (double*)malloc(sizeof(double) * d_in);
+  for (i64 p = 0; p < d_in; ++p)
+    for (i64 k = 0; k < d_in; ++k)
+      Ht[p * d_in + k] = a_full[p] * (double)H[p * d_in + k] * a_full[k];
+  for (i64 i = 0; i < d_in; ++i) z[i] = (double)q[i] - (w[i] - b_full[i]) / a_full[i];
+  for (i64 p = 0; p < d_in; ++p) {
+    double acc = 0.0;
+    for (i64 k = 0; k < d_in; ++k) acc = acc + Ht[p * d_in + k] * z[k];
+    gt[p] = 2.0 * acc;
+  }
+  i64 moves = 0;
+  for (i64 t = 0; t < T; ++t) {
+    double best = 0.0;
+    i64 bi = -1;
+    int br = 0;
+    for (i64 i = 0; i < d_in; ++i)
+      for (int r = 0; r <= L; ++r) {
+        const double dr = (double)(r - (int)q[i]);
+        if (dr == 0.0) continue;
+        const double delta = dr * dr * Ht[i * d_in + i] + dr * gt[i];
+        if (delta < best) { best = delta; bi = i; br = r; }
+      }
+    if (bi < 0) break;
+    const double dr = (double)(br - (int)q[bi]);
+    for (i64 p = 0; p < d_in; ++p) gt[p] = gt[p] + 2.0 * dr * Ht[bi * d_in + p];
+    q[bi] = (uint8_t)br;
+    if (trace_i) { trace_i[moves] = (int)bi; trace_r[moves] = br; }
+    ++moves;
+  }
+  free(Ht); free(gt); free(z);
+  return moves;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Layer loss sum_j e_j^T H e_j (Eq. 1 expanded with H = X^T X).             */
+/* per_col (may be NULL): [d_out].  Returns the total through *total.        */
+/* ------------------------------------------------------------------------ */
+int cdqo_layer_loss(const float* H, const double* W, i64 d_in, i64 d_out,
+                    i64 group_size, const float* scale, const float* zero,
+                    const uint8_t* Q, double* per_col, double* total) {
+  if (!H || !W || !scale || !zero || !Q || !total) return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g) return 2;
+  const i64 ng = d_in / g;
+  double* col_loss = (double*)malloc(sizeof(double) * d_out);
+#pragma omp parallel
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    double* he = (double*)malloc(sizeof(double) * d_in);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) { w[i] = W[i * d_out + j]; q[i] = Q[i * d_out + j]; }
+      for (i64 t = 0; t < ng; ++t) { a[t] = scale[t * d_out + j]; b[t] = zero[t * d_out + j]; }
+      residual(w, q, a, b, d_in, g, e);
+      col_loss[j] = quad_form(H, e, d_in, he);
+    }
+    free(w); free(e); free(he); free(q); free(a); free(b);
+  }
+  double sum = 0.0;
+  for (i64 j = 0; j < d_out; ++j) sum = sum + col_loss[j]; /* ascending j */
+  if (per_col) memcpy(per_col, col_loss, sizeof(double) * d_out);
+  *total = sum;
+  free(col_loss);
+  return 0;
+}
