@@ -1,0 +1,171 @@
+/*
+ * cdq.h -- C ABI of the B200 (sm_100a) CDQuant hot path.
+ *
+ * Post-training weight quantization by greedy coordinate descent on the
+ * layer-wise reconstruction loss ||X (W - W_hat)||_F^2 (paper, Section 3,
+ * Eq. 1).  Every output column of W is an independent descent problem; all of
+ * them share one Hessian H = X^T X.
+ *
+ * Notation (paper, Section 3 "Notation"):
+ *   X      [n, d_in]      calibration inputs, row-major
+ *   W      [d_in, d_out]  layer weights, row-major with leading dimension ldw
+ *   H      [d_in, d_in]   X^T X, fp32, both triangles stored
+ *   c      bits; levels are 0 .. 2^c - 1
+ *   Q      [d_in, d_out]  codes, one byte each, row-major, dense
+ *   a, b   scale and zero, [d_in/g, d_out] fp32 row-major (one row when
+ *          per-channel); W_hat[i,j] = a[i/g,j] * Q[i,j] + b[i/g,j]
+ *
+ * General rules
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless the
+ *     argument is marked "host".  The library allocates no device memory:
+ *     scratch comes from the caller's workspace `ws` (size from
+ *     cdq_workspace_bytes, 256-byte aligned).  A too-small workspace gives
+ *     CDQ_ERR_WORKSPACE before anything is launched.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work, except where a host result is returned
+ *     (cdq_cd_solve with stats != NULL, cdq_layer_loss with loss != NULL):
+ *     those synchronise `stream` before returning.
+ *   - Errors are returned as status codes; nothing aborts or throws.
+ *     Arguments are validated before any launch.  A device-side wait that
+ *     exceeds its bound is reported as CDQ_ERR_TIMEOUT by the next call that
+ *     synchronises (cdq_last_device_status reads it explicitly).
+ *   - Two arithmetic modes.  CDQ_MODE_FAST is the production path: fp32 H,
+ *     fp32 candidate scoring, gradient kept in fp64, tensor cores for the
+ *     Hessian.  CDQ_MODE_FP64_VERIFY runs plain fp64 kernels that follow a
+ *     fixed summation order (ascending index, no fused multiply-add) so that
+ *     codes can be compared bit for bit with a CPU implementation of the same
+ *     steps; it is meant for small layers.
+ */
+#ifndef CDQ_H_
+#define CDQ_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CDQ_OK = 0,
+  CDQ_ERR_INVALID_ARG = 1, /* null pointer, bad enum, bits outside 1..8, ...    */
+  CDQ_ERR_SHAPE = 2,       /* non-positive size, d_in % group_size != 0, ld too small */
+  CDQ_ERR_UNSUPPORTED = 3, /* valid request this build has no kernel for       */
+  CDQ_ERR_WORKSPACE = 4,   /* ws NULL / misaligned / smaller than required      */
+  CDQ_ERR_CUDA = 5,        /* a CUDA runtime call failed                        */
+  CDQ_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out                */
+} cdq_status;
+
+typedef enum { CDQ_F32 = 0, CDQ_BF16 = 1 } cdq_dtype;
+typedef enum { CDQ_MODE_FAST = 0, CDQ_MODE_FP64_VERIFY = 1 } cdq_mode;
+
+/* Which entry point a workspace size is asked for. */
+typedef enum {
+  CDQ_CALL_HESSIAN = 0,
+  CDQ_CALL_INIT_RTN = 1,
+  CDQ_CALL_CD_SOLVE = 2,
+  CDQ_CALL_LAYER_LOSS = 3
+} cdq_call;
+
+/* Quantization grid (paper: c in "Notation"; group size g in the sub-channel
+ * section; clipping grid Gamma in the OWC paragraph after Eq. 2). */
+typedef struct {
+  int bits;       /* c, 1..8 */
+  int group_size; /* g along d_in; 0 => per-channel (g = d_in); d_in % g == 0 */
+  int n_clip;     /* |Gamma|; <= 1 => MinMax (gamma = 1) */
+  float clip_lo;  /* Gamma = { lo + (hi-lo)*k/(n_clip-1), k = 0..n_clip-1 } */
+  float clip_hi;
+} cdq_grid_desc;
+
+typedef struct {
+  unsigned long long steps;             /* step budget: passes * d_in * d_out            */
+  unsigned long long committed;         /* moves actually made                           */
+  unsigned long long columns_converged; /* columns that ran out of improving moves       */
+  double loss_before;                   /* sum_j e_j^T H e_j at entry (from G0)          */
+  double loss_after;                    /* loss_before + sum of committed decreases      */
+} cdq_cd_stats;
+
+/*
+ * H = X^T X  (paper: Section 3 "Notation"; Algorithm 1 line 2), plus the
+ * optional regulariser of Section 4: H_ii += lambda_rel * mean(diag H).
+ *   X          [n, d_in] of type xt, leading dimension ldx (elements, >= d_in).
+ *              BF16 input additionally needs X 16-byte aligned and ldx % 8 == 0.
+ *   accumulate 0: H is overwritten.  1: H += X^T X (calibration rows arriving
+ *              in chunks); lambda_rel must then be 0 except on the last chunk.
+ *   H          [d_in, d_in] fp32 out (in/out when accumulating).
+ * FAST: bf16 inputs run on the tensor cores (fp32 accumulation); fp32 inputs
+ * use an fp64-accumulating SIMT kernel.  VERIFY: every entry is the ascending-k
+ * fp64 sum, rounded once to fp32; accumulate is not supported there.
+ */
+cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in, long long ldx,
+                       float lambda_rel, int accumulate, float* H, cdq_mode mode, void* ws,
+                       size_t ws_bytes, void* stream);
+
+/*
+ * Grid and round-to-nearest codes (paper: Eq. 2; gamma = 1 is MinMax), with
+ * the Optimal Weight Clipping search when grid->n_clip > 1 (paper: the
+ * minimisation over gamma stated after Eq. 2, solved by grid search).
+ * Per column j and group t: b = min(w), a = gamma * (max(w) - min(w)) / (2^c - 1),
+ * q = clamp(round_half_even((w - b) / a), 0, 2^c - 1); a constant group gets
+ * a = 0 and all-zero codes.  With n_clip > 1, one gamma per output column is
+ * applied to every group of the column and is the grid point with the
+ * smallest column loss e^T H e (lowest index on ties).
+ *   W          [d_in, d_out] of type wt, leading dimension ldw.
+ *   H          [d_in, d_in] fp32; may be NULL iff n_clip <= 1.
+ *   scale,zero [d_in/g, d_out] fp32 out.
+ *   Q          [d_in, d_out] u8 out.
+ *   gamma_out  [d_out] fp32 out, chosen clipping strength; may be NULL.
+ * The rounding decision is taken in fp64 in both modes.
+ */
+cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                        const float* H, const cdq_grid_desc* grid, float* scale, float* zero,
+                        unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws,
+                        size_t ws_bytes, void* stream);
+
+/*
+ * Greedy coordinate descent on every column (paper: Algorithm 1; Algorithm 4
+ * for sub-channel grids), T = passes * d_in steps per column at most.
+ * Weight-unit form of the iteration: G = 2 H (W_hat - W); a move of
+ * coordinate i to level r changes the loss by d^2 H_ii + d G_i with
+ * d = a_i (r - q_i); the move with the most negative change is made (ties:
+ * lowest i, then lowest r); G += 2 d H[i,:].  A column stops early when no
+ * move lowers its loss.
+ *   Q      in: initial codes q0 (e.g. from cdq_init_rtn); out: result.
+ *   stats  host pointer, may be NULL (then the call does not synchronise).
+ * FAST: scoring in fp32 from an fp64 gradient; VERIFY: fp64 level scan in the
+ * fixed order, bit-reproducible.
+ */
+cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                        long long ldw, const cdq_grid_desc* grid, const float* scale,
+                        const float* zero, unsigned char* Q, int passes, cdq_mode mode,
+                        cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Layer loss sum_j e_j^T H e_j with e = W_hat - W (paper: Eq. 1 written with
+ * H = X^T X; the objective value the paper reports for a solution).
+ *   loss     host pointer to one double, may be NULL.
+ *   per_col  [d_out] fp64 device out, may be NULL.
+ */
+cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                          long long ldw, const cdq_grid_desc* grid, const float* scale,
+                          const float* zero, const unsigned char* Q, double* loss, double* per_col,
+                          cdq_mode mode, void* ws, size_t ws_bytes, void* stream);
+
+/* Bytes of workspace `which` needs for these sizes (n is used by the Hessian only). */
+size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long long d_out,
+                           const cdq_grid_desc* grid, cdq_mode mode);
+
+/* Reads and clears the device-side status word (synchronises the device). */
+cdq_status cdq_last_device_status(void);
+
+/* Text of the most recent CDQ_ERR_CUDA in this process (CUDA error name, the failing step);
+ * an empty string if there was none.  The pointer stays valid; the text is overwritten by
+ * the next such error. */
+const char* cdq_last_error_detail(void);
+
+const char* cdq_status_string(cdq_status s);
+int cdq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CDQ_H_ */

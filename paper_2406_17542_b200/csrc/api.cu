@@ -1,0 +1,306 @@
+// extern "C" entry points declared in include/cdq.h: argument validation, workspace
+// carving and kernel sequencing.  No device memory is allocated here.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace cdq {
+
+__device__ int g_device_status = 0;
+
+int* device_status_word() {
+  int* p = nullptr;
+  if (cudaGetSymbolAddress((void**)&p, g_device_status) != cudaSuccess) return nullptr;
+  return p;
+}
+
+namespace {
+
+bool valid_dtype(cdq_dtype t) { return t == CDQ_F32 || t == CDQ_BF16; }
+bool valid_mode(cdq_mode m) { return m == CDQ_MODE_FAST || m == CDQ_MODE_FP64_VERIFY; }
+
+cdq_status check_grid(const cdq_grid_desc* g, long long d_in) {
+  if (!g) return CDQ_ERR_INVALID_ARG;
+  if (g->bits < 1 || g->bits > 8) return CDQ_ERR_INVALID_ARG;
+  if (g->group_size < 0) return CDQ_ERR_INVALID_ARG;
+  if (g->n_clip > 256) return CDQ_ERR_INVALID_ARG;
+  if (g->n_clip > 1 && !(g->clip_lo > 0.f && g->clip_hi >= g->clip_lo)) return CDQ_ERR_INVALID_ARG;
+  if (g->group_size > 0 && d_in % g->group_size) return CDQ_ERR_SHAPE;
+  return CDQ_OK;
+}
+
+cdq_status check_ws(const void* ws, size_t have, size_t need) {
+  if (need == 0) return CDQ_OK;
+  if (!ws || ((uintptr_t)ws % kAlign) || have < need) return CDQ_ERR_WORKSPACE;
+  return CDQ_OK;
+}
+
+cdq_status check_layer_shape(long long d_in, long long d_out, long long ldw) {
+  if (d_in < 1 || d_out < 1 || ldw < d_out) return CDQ_ERR_SHAPE;
+  if (d_in > 65535) return CDQ_ERR_UNSUPPORTED;  // rows index a grid dimension
+  if (d_out > 2147483647LL / 2) return CDQ_ERR_UNSUPPORTED;
+  return CDQ_OK;
+}
+
+Layer make_layer(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                 const cdq_grid_desc* grid, const float* scale, const float* zero) {
+  Layer ly{};
+  ly.H = H; ly.W = W; ly.wt = wt; ly.d_in = d_in; ly.d_out = d_out; ly.ldw = ldw;
+  ly.bits = grid->bits; ly.L = (1 << grid->bits) - 1;
+  ly.g = grid->group_size > 0 ? grid->group_size : d_in;
+  ly.ng = d_in / ly.g;
+  ly.scale = scale; ly.zero = zero;
+  return ly;
+}
+
+// Workspace of cdq_cd_solve / cdq_layer_loss.
+struct SolveWs {
+  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, total;
+  long long ldg, d_pad;
+};
+SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd) {
+  SolveWs w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  w.ldg = (d_in + 3) / 4 * 4;
+  w.d_pad = cd_fast_pad(d_in);
+  w.E = take(sizeof(double) * d_in * d_out);
+  if (with_cd) {
+    w.G = take(sizeof(double) * d_out * w.ldg);
+    w.Qt = take((size_t)d_out * d_in);
+    w.hdiag = take(sizeof(float) * w.d_pad);
+    w.half_inv = take(sizeof(float) * w.d_pad);
+  }
+  w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
+  w.col_loss = take(sizeof(double) * d_out);
+  w.scalars = take(256);  // [0]: double loss sum; [64..): CdCounters
+  w.total = off;
+  return w;
+}
+
+ResidualSrc codes_src(const Layer& ly, const unsigned char* Q) {
+  ResidualSrc s{};
+  s.W = ly.W; s.wt = ly.wt; s.ldw = ly.ldw; s.scale = ly.scale; s.zero = ly.zero; s.Q = Q;
+  s.use_gamma = 0; s.L = ly.L; s.g = ly.g; s.d_out = ly.d_out;
+  return s;
+}
+
+char g_error_detail[256] = "";
+
+void note_cuda_error(cudaError_t e, const char* what, int line) {
+  snprintf(g_error_detail, sizeof(g_error_detail), "%s (%s) at api.cu:%d: %s", cudaGetErrorName(e),
+           cudaGetErrorString(e), line, what);
+}
+
+// CDQ_DEBUG_SYNC=1 in the environment synchronises the device after every step, so that an
+// asynchronous kernel failure is attributed to the step that caused it.
+bool debug_sync() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("CDQ_DEBUG_SYNC");
+    v = (e && e[0] == '1') ? 1 : 0;
+  }
+  return v == 1;
+}
+
+#define CDQ_CUDA(expr)                                  \
+  do {                                                  \
+    cudaError_t _e = (expr);                            \
+    if (_e == cudaSuccess && debug_sync()) _e = cudaDeviceSynchronize(); \
+    if (_e != cudaSuccess) {                            \
+      note_cuda_error(_e, #expr, __LINE__);             \
+      return CDQ_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+cdq_status read_device_status_after_sync() {
+  int flag = 0;
+  if (cudaMemcpyFromSymbol(&flag, g_device_status, sizeof(int)) != cudaSuccess) return CDQ_ERR_CUDA;
+  if (flag == kFlagOk) return CDQ_OK;
+  int zero = 0;
+  cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+  return CDQ_ERR_TIMEOUT;
+}
+
+}  // namespace
+}  // namespace cdq
+
+using namespace cdq;
+
+extern "C" {
+
+int cdq_version(void) { return 100; }
+
+const char* cdq_status_string(cdq_status s) {
+  switch (s) {
+    case CDQ_OK: return "ok";
+    case CDQ_ERR_INVALID_ARG: return "invalid argument";
+    case CDQ_ERR_SHAPE: return "bad shape";
+    case CDQ_ERR_UNSUPPORTED: return "unsupported";
+    case CDQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CDQ_ERR_CUDA: return "CUDA runtime error";
+    case CDQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+const char* cdq_last_error_detail(void) { return g_error_detail; }
+
+cdq_status cdq_last_device_status(void) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return CDQ_ERR_CUDA;
+  return read_device_status_after_sync();
+}
+
+size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long long d_out, const cdq_grid_desc* grid,
+                           cdq_mode mode) {
+  if (d_in < 1) return 0;
+  switch (which) {
+    case CDQ_CALL_HESSIAN:
+      if (mode == CDQ_MODE_FP64_VERIFY) return align_up(sizeof(double) * d_in * d_in);
+      return hessian_tc_workspace(n, d_in);
+    case CDQ_CALL_INIT_RTN: {
+      if (!grid || d_out < 1) return 0;
+      const long long g = grid->group_size > 0 ? grid->group_size : d_in;
+      if (g < 1 || d_in % g) return 0;
+      return init_rtn_workspace(d_in, d_out, g, grid->n_clip, mode);
+    }
+    case CDQ_CALL_CD_SOLVE:
+      if (d_out < 1) return 0;
+      return solve_ws_layout(d_in, d_out, mode, true).total;
+    case CDQ_CALL_LAYER_LOSS:
+      if (d_out < 1) return 0;
+      return solve_ws_layout(d_in, d_out, mode, false).total;
+  }
+  return 0;
+}
+
+cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in, long long ldx, float lambda_rel,
+                       int accumulate, float* H, cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {
+  if (!X || !H || !valid_dtype(xt) || !valid_mode(mode) || !(lambda_rel >= 0.f)) return CDQ_ERR_INVALID_ARG;
+  if (n < 1 || d_in < 1 || ldx < d_in) return CDQ_ERR_SHAPE;
+  if (d_in > 65535) return CDQ_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (mode == CDQ_MODE_FP64_VERIFY) {
+    if (accumulate) return CDQ_ERR_UNSUPPORTED;
+    cdq_status s = check_ws(ws, ws_bytes, align_up(sizeof(double) * d_in * d_in));
+    if (s != CDQ_OK) return s;
+    CDQ_CUDA(launch_hessian_verify(X, xt, n, d_in, ldx, (double)lambda_rel, H, (double*)ws, st));
+    return CDQ_OK;
+  }
+  if (xt == CDQ_BF16 && hessian_tc_supported(n, d_in, ldx, X)) {
+    cdq_status s = check_ws(ws, ws_bytes, hessian_tc_workspace(n, d_in));
+    if (s != CDQ_OK) return s;
+    CDQ_CUDA(launch_hessian_tc(X, n, d_in, ldx, accumulate, H, ws, st));
+  } else {
+    CDQ_CUDA(launch_hessian_simt(X, xt, n, d_in, ldx, accumulate, H, st));
+  }
+  if (lambda_rel > 0.f) CDQ_CUDA(launch_hessian_lambda(H, d_in, (double)lambda_rel, nullptr, st));
+  return CDQ_OK;
+}
+
+cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw, const float* H,
+                        const cdq_grid_desc* grid, float* scale, float* zero, unsigned char* Q, float* gamma_out,
+                        cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {
+  if (!W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode)) return CDQ_ERR_INVALID_ARG;
+  cdq_status s = check_layer_shape(d_in, d_out, ldw);
+  if (s != CDQ_OK) return s;
+  s = check_grid(grid, d_in);
+  if (s != CDQ_OK) return s;
+  if (grid->n_clip > 1 && !H) return CDQ_ERR_INVALID_ARG;
+  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, nullptr, nullptr);
+  if (ly.ng > 65535) return CDQ_ERR_UNSUPPORTED;
+  s = check_ws(ws, ws_bytes, init_rtn_workspace(d_in, d_out, ly.g, grid->n_clip, mode));
+  if (s != CDQ_OK) return s;
+  CDQ_CUDA(launch_init_rtn(ly, *grid, scale, zero, Q, gamma_out, mode, ws, (cudaStream_t)stream));
+  return CDQ_OK;
+}
+
+cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                        const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
+                        int passes, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
+  if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || passes < 0)
+    return CDQ_ERR_INVALID_ARG;
+  cdq_status s = check_layer_shape(d_in, d_out, ldw);
+  if (s != CDQ_OK) return s;
+  s = check_grid(grid, d_in);
+  if (s != CDQ_OK) return s;
+  if (mode == CDQ_MODE_FAST && !cd_fast_supported(d_in)) return CDQ_ERR_UNSUPPORTED;
+  const SolveWs L = solve_ws_layout(d_in, d_out, mode, true);
+  s = check_ws(ws, ws_bytes, L.total);
+  if (s != CDQ_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, scale, zero);
+  char* base = (char*)ws;
+  double* E = (double*)(base + L.E);
+  double* G = (double*)(base + L.G);
+  unsigned char* Qt = (unsigned char*)(base + L.Qt);
+  float* hdiag = (float*)(base + L.hdiag);
+  float* half_inv = (float*)(base + L.half_inv);
+  double* part = (double*)(base + L.part);
+  double* col_loss = (double*)(base + L.col_loss);
+  double* loss_sum = (double*)(base + L.scalars);
+  CdCounters* ctr = (CdCounters*)(base + L.scalars + 64);
+  const long long steps_per_col = (long long)passes * d_in;
+
+  // G0 = 2 H (W_hat - W) and the loss at entry
+  CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
+  if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, G, L.ldg, col_loss, part, st));
+  else CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, G, L.ldg, col_loss, st));
+  CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
+  CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, Qt, st));
+  CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
+  if (mode == CDQ_MODE_FAST) {
+    CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
+    CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, hdiag, half_inv, steps_per_col, ctr, st));
+  } else {
+    CDQ_CUDA(launch_cd_verify(ly, G, L.ldg, Qt, steps_per_col, ctr, st));
+  }
+  CDQ_CUDA(launch_transpose_u8(Qt, d_out, d_in, Q, st));
+  if (stats) {
+    CdCounters hc;
+    double lb = 0.0;
+    CDQ_CUDA(cudaMemcpyAsync(&hc, ctr, sizeof(CdCounters), cudaMemcpyDeviceToHost, st));
+    CDQ_CUDA(cudaMemcpyAsync(&lb, loss_sum, sizeof(double), cudaMemcpyDeviceToHost, st));
+    CDQ_CUDA(cudaStreamSynchronize(st));
+    stats->steps = (unsigned long long)steps_per_col * (unsigned long long)d_out;
+    stats->committed = hc.committed;
+    stats->columns_converged = hc.converged;
+    stats->loss_before = lb;
+    stats->loss_after = lb + hc.delta_sum;
+    return read_device_status_after_sync();
+  }
+  return CDQ_OK;
+}
+
+cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                          const cdq_grid_desc* grid, const float* scale, const float* zero, const unsigned char* Q,
+                          double* loss, double* per_col, cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {
+  if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode)) return CDQ_ERR_INVALID_ARG;
+  cdq_status s = check_layer_shape(d_in, d_out, ldw);
+  if (s != CDQ_OK) return s;
+  s = check_grid(grid, d_in);
+  if (s != CDQ_OK) return s;
+  const SolveWs L = solve_ws_layout(d_in, d_out, mode, false);
+  s = check_ws(ws, ws_bytes, L.total);
+  if (s != CDQ_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, scale, zero);
+  char* base = (char*)ws;
+  double* E = (double*)(base + L.E);
+  double* part = (double*)(base + L.part);
+  double* col_loss = per_col ? per_col : (double*)(base + L.col_loss);
+  double* loss_sum = (double*)(base + L.scalars);
+  CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
+  if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, nullptr, 0, col_loss, part, st));
+  else CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, nullptr, 0, col_loss, st));
+  if (loss) {
+    CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
+    CDQ_CUDA(cudaMemcpyAsync(loss, loss_sum, sizeof(double), cudaMemcpyDeviceToHost, st));
+    CDQ_CUDA(cudaStreamSynchronize(st));
+  }
+  return CDQ_OK;
+}
+
+}  // extern "C"

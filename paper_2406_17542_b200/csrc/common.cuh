@@ -1,0 +1,102 @@
+// Shared declarations of the CUDA library behind include/cdq.h.
+// Everything here is internal; the only exported symbols are the extern "C"
+// entry points in api.cu.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/cdq.h"
+
+namespace cdq {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+// Device status word: kernels with bounded waits record a failure here.
+enum DeviceFlag : int { kFlagOk = 0, kFlagWaitTimeout = 1 };
+int* device_status_word();  // device address of the status word (per process)
+
+// Resolved problem description shared by the launchers.
+struct Layer {
+  const float* H;
+  const void* W;
+  cdq_dtype wt;
+  long long d_in, d_out, ldw;
+  int bits, L;
+  long long g;   // group size actually used (d_in when per-channel)
+  long long ng;  // d_in / g
+  const float* scale;
+  const float* zero;
+};
+
+// Load one weight as double (exact widening).
+__device__ __forceinline__ double load_w(const void* W, cdq_dtype wt, long long idx) {
+  if (wt == CDQ_BF16) return (double)__bfloat162float(((const __nv_bfloat16*)W)[idx]);
+  return (double)((const float*)W)[idx];
+}
+
+// ---- launchers (one per .cu file) -----------------------------------------
+// hessian_simt.cu
+cudaError_t launch_hessian_verify(const void* X, cdq_dtype xt, long long n, long long d_in, long long ldx,
+                                  double lambda_rel, float* H, double* H64, cudaStream_t st);
+cudaError_t launch_hessian_simt(const void* X, cdq_dtype xt, long long n, long long d_in, long long ldx,
+                                int accumulate, float* H, cudaStream_t st);
+cudaError_t launch_hessian_lambda(float* H, long long d_in, double lambda_rel, double* scratch, cudaStream_t st);
+
+// hessian_tc.cu (tcgen05 / TMEM / TMA path for bf16 inputs)
+bool hessian_tc_supported(long long n, long long d_in, long long ldx, const void* X);
+size_t hessian_tc_workspace(long long n, long long d_in);
+cudaError_t launch_hessian_tc(const void* X, long long n, long long d_in, long long ldx, int accumulate,
+                              float* H, void* ws, cudaStream_t st);
+
+// init_rtn.cu
+size_t init_rtn_workspace(long long d_in, long long d_out, long long g, int n_clip, cdq_mode mode);
+cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* scale, float* zero,
+                            unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws, cudaStream_t st);
+
+// Residual E = W_hat - W in fp64, [d_in, d_out] row-major, either from stored codes or, for
+// the OWC search, from per-group min/max and one clipping strength (codes formed on the fly).
+struct ResidualSrc {
+  const void* W; cdq_dtype wt; long long ldw;
+  const float* scale; const float* zero; const unsigned char* Q;  // codes path
+  const float* mn; const float* mx; double gamma; int L; int use_gamma;  // OWC path
+  long long g, d_out;
+};
+cudaError_t launch_residual_f64(const ResidualSrc& src, long long d_in, double* E, cudaStream_t st);
+
+// gemm_f64.cu : C = H * E in fp64.
+// G (may be NULL): [d_out, ldg] doubles, G[j][p] = 2 * C[p][j].
+// col_loss (may be NULL): [d_out] doubles, e_j^T H e_j = sum_p E[p][j] C[p][j]; needs the
+// scratch `part` of gemm_partials_elems(d_in, d_out) doubles.
+size_t gemm_partials_elems(long long d_in, long long d_out);
+cudaError_t launch_gemm_he(const float* H, long long d_in, long long d_out, const double* E,
+                           double* G, long long ldg, double* col_loss, double* part, cudaStream_t st);
+// fixed-order version (ascending k, no fused multiply-add)
+// C: scratch of d_in * d_out doubles.
+cudaError_t launch_gemm_he_verify(const float* H, long long d_in, long long d_out, const double* E, double* C,
+                                  double* G, long long ldg, double* col_loss, cudaStream_t st);
+
+// cd_kernel.cu
+struct CdCounters {            // lives in the workspace, zeroed by the launcher
+  unsigned long long committed;
+  unsigned long long converged;
+  double delta_sum;
+  int next_col;
+  int pad;
+};
+cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols,
+                                unsigned char* dst, cudaStream_t st);  // dst[c][r] = src[r][c]
+long long cd_fast_pad(long long d_in);      // padded length of hdiag / half_inv
+bool cd_fast_supported(long long d_in);
+cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* half_inv,
+                        cudaStream_t st);
+cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt,
+                           const float* hdiag, const float* half_inv, long long steps_per_col,
+                           CdCounters* ctr, cudaStream_t st);
+cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt,
+                             long long steps_per_col, CdCounters* ctr, cudaStream_t st);
+cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st);  // ascending order
+
+}  // namespace cdq
