@@ -42,7 +42,7 @@ class cdq_grid_desc(ctypes.Structure):
 class cdq_cd_stats(ctypes.Structure):
     _fields_ = [("steps", ctypes.c_ulonglong), ("committed", ctypes.c_ulonglong),
                 ("columns_converged", ctypes.c_ulonglong), ("loss_before", ctypes.c_double),
-                ("loss_after", ctypes.c_double)]
+                ("loss_after", ctypes.c_double), ("kernel_ms", ctypes.c_double)]
 
 
 @dataclass
@@ -196,7 +196,7 @@ def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tens
     if not want_stats:
         return None
     return {"steps": stats.steps, "committed": stats.committed, "columns_converged": stats.columns_converged,
-            "loss_before": stats.loss_before, "loss_after": stats.loss_after}
+            "loss_before": stats.loss_before, "loss_after": stats.loss_after, "kernel_ms": stats.kernel_ms}
 
 
 def cdq_layer_loss(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,

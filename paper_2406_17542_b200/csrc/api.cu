@@ -251,12 +251,20 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
   CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, Qt, st));
   CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (stats) {
+    CDQ_CUDA(cudaEventCreate(&ev0));
+    CDQ_CUDA(cudaEventCreate(&ev1));
+  }
   if (mode == CDQ_MODE_FAST) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
+    if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
     CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, hdiag, half_inv, steps_per_col, ctr, st));
   } else {
+    if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
     CDQ_CUDA(launch_cd_verify(ly, G, L.ldg, Qt, steps_per_col, ctr, st));
   }
+  if (stats) CDQ_CUDA(cudaEventRecord(ev1, st));
   CDQ_CUDA(launch_transpose_u8(Qt, d_out, d_in, Q, st));
   if (stats) {
     CdCounters hc;
@@ -269,6 +277,11 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
     stats->columns_converged = hc.converged;
     stats->loss_before = lb;
     stats->loss_after = lb + hc.delta_sum;
+    float ms = 0.f;
+    CDQ_CUDA(cudaEventElapsedTime(&ms, ev0, ev1));
+    stats->kernel_ms = (double)ms;
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
     return read_device_status_after_sync();
   }
   return CDQ_OK;
