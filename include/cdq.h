@@ -152,6 +152,40 @@ cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long
                           const float* zero, const unsigned char* Q, double* loss, double* per_col,
                           cdq_mode mode, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * The layer loss for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of cdq_layer_loss, same result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region whose memory
+ * was handed out up front and is now frozen (a serving process after start-up, a plugin
+ * inside another framework's memory pool that does not lend scratch), or a latency-critical
+ * path where an allocation could block on the driver.  Such a caller cannot provide the
+ * workspace that cdq_layer_loss asks for, so this entry point brings its own: a fixed array
+ * of CDQ_STATIC_SCRATCH_BYTES that is part of the library image.  Every GPU on which the
+ * library is used holds that much memory from the first use until the process exits.
+ *
+ *   Arguments as for cdq_layer_loss, FAST arithmetic, no workspace.  Inputs and outputs are
+ *   still the caller's: H, W, scale, zero, Q and per_col are device pointers, loss is a host
+ *   pointer (the call synchronises `stream` when loss != NULL).
+ *   Limit: 8 * d_in * d_out bytes for the residual plus about 8 * d_out * (d_in / 128 + 2)
+ *   must fit in the array (e.g. 2048 x 1024 or 1024 x 2048); a larger layer is rejected with
+ *   CDQ_ERR_WORKSPACE before anything is launched, and cdq_last_error_detail() says how
+ *   much was needed.
+ *   The call itself allocates and frees nothing, on the host side of the runtime included
+ *   (no cudaMalloc / cudaFree, no allocating library routine).
+ *   First call on a device: it looks up the device address of the array (the device must be
+ *   current).  Make that first call during set-up, before any stream capture is begun.
+ *   All calls on one GPU share the one array, and it keeps the previous call's contents.
+ *   Nothing in it has to start at zero -- each call overwrites every region before reading
+ *   it -- but two calls that overlap on the GPU (different streams, or different host threads
+ *   on different streams) race on it: serialise them.
+ */
+#define CDQ_STATIC_SCRATCH_BYTES (20u * 1024u * 1024u)
+cdq_status cdq_layer_loss_static(const float* H, const void* W, cdq_dtype wt, long long d_in,
+                                 long long d_out, long long ldw, const cdq_grid_desc* grid,
+                                 const float* scale, const float* zero, const unsigned char* Q,
+                                 double* loss, double* per_col, void* stream);
+
 /* Bytes of workspace `which` needs for these sizes (n is used by the Hessian only). */
 size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long long d_out,
                            const cdq_grid_desc* grid, cdq_mode mode);
@@ -159,8 +193,8 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
 /* Reads and clears the device-side status word (synchronises the device). */
 cdq_status cdq_last_device_status(void);
 
-/* Text of the most recent CDQ_ERR_CUDA in this process (CUDA error name, the failing step);
- * an empty string if there was none.  The pointer stays valid; the text is overwritten by
+/* Text of the most recent CDQ_ERR_CUDA in this process (CUDA error name, the failing step),
+ * or of a size rejection by cdq_layer_loss_static; an empty string if there was none.  The pointer stays valid; the text is overwritten by
  * the next such error. */
 const char* cdq_last_error_detail(void);
 

@@ -24,7 +24,8 @@ MODE_FAST, MODE_FP64_VERIFY = 0, 1
 CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS = 0, 1, 2, 3
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_cd_solve", "cdq_layer_loss", "cdq_workspace_bytes",
+EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_cd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
+           "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version"]
 
 
@@ -83,6 +84,8 @@ def load():
     lib.cdq_cd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_layer_loss.restype = ci
     lib.cdq_layer_loss.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ctypes.POINTER(ctypes.c_double), vp, ci, vp, sz, vp]
+    lib.cdq_layer_loss_static.restype = ci
+    lib.cdq_layer_loss_static.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ctypes.POINTER(ctypes.c_double), vp, vp]
     _lib = lib
     return lib
 
@@ -214,6 +217,34 @@ def cdq_layer_loss(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Te
                                pc.data_ptr() if pc is not None else None, _MODES[mode], wptr, wbytes, _stream())
     _check(st, "cdq_layer_loss")
     return (loss.value, pc) if per_col else loss.value
+
+
+STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
+
+
+def cdq_layer_loss_static(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,
+                          Q: torch.Tensor, per_col: torch.Tensor | None = None) -> float:
+    """The layer loss without a workspace: for callers that may not allocate device memory (a
+    frozen memory pool, a latency-critical path).  Scratch is a fixed STATIC_SCRATCH_BYTES
+    array inside the library, shared by all calls on a GPU, so calls must not overlap; layers
+    whose residual does not fit are refused with CDQ_ERR_WORKSPACE.  `per_col` (fp64 [d_out]
+    on the device), if given, receives the per-column losses -- this binding allocates nothing
+    either.  The first call on a device should happen during set-up."""
+    d_in, d_out = W.shape
+    gd = grid.c()
+    loss = ctypes.c_double(0.0)
+    st = load().cdq_layer_loss_static(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0),
+                                      ctypes.byref(gd), scale.data_ptr(), zero.data_ptr(), Q.data_ptr(),
+                                      ctypes.byref(loss), per_col.data_ptr() if per_col is not None else None,
+                                      _stream())
+    if status_is_workspace(st):
+        raise CdqError(st, "cdq_layer_loss_static [" + load().cdq_last_error_detail().decode() + "]")
+    _check(st, "cdq_layer_loss_static")
+    return loss.value
+
+
+def status_is_workspace(st: int) -> bool:
+    return st == 4
 
 
 def quantize_layer(X: torch.Tensor, W: torch.Tensor, grid: Grid, passes: int, lambda_rel: float = 0.0, mode="fast",

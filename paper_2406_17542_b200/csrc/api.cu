@@ -16,6 +16,9 @@ int* device_status_word() {
   return p;
 }
 
+static char g_error_detail[256] = "";
+void set_error_detail(const char* text) { snprintf(g_error_detail, sizeof(g_error_detail), "%s", text); }
+
 namespace {
 
 bool valid_dtype(cdq_dtype t) { return t == CDQ_F32 || t == CDQ_BF16; }
@@ -86,8 +89,6 @@ ResidualSrc codes_src(const Layer& ly, const unsigned char* Q) {
   s.use_gamma = 0; s.L = ly.L; s.g = ly.g; s.d_out = ly.d_out;
   return s;
 }
-
-char g_error_detail[256] = "";
 
 void note_cuda_error(cudaError_t e, const char* what, int line) {
   snprintf(g_error_detail, sizeof(g_error_detail), "%s (%s) at api.cu:%d: %s", cudaGetErrorName(e),

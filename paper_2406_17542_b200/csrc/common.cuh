@@ -18,6 +18,9 @@ inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a
 enum DeviceFlag : int { kFlagOk = 0, kFlagWaitTimeout = 1 };
 int* device_status_word();  // device address of the status word (per process)
 
+// Text returned by cdq_last_error_detail().
+void set_error_detail(const char* text);
+
 // Resolved problem description shared by the launchers.
 struct Layer {
   const float* H;
