@@ -57,7 +57,7 @@ def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
         list(ex.map(run, jobs))
     objs = [os.path.join(OBJ, s.replace(".cu", ".o")) for s in SOURCES]
     if jobs or not os.path.exists(LIB):
-        run([nvcc, "-shared", "-o", LIB, *objs, "-lcuda"])
+        run([nvcc, "-shared", "-o", LIB, *objs])
     return LIB
 
 

@@ -138,3 +138,29 @@ def test_resume_from_previous_codes():
     s2 = B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, 1)
     assert s2["committed"] == 0 and s2["columns_converged"] == cfg.d_out
     np.testing.assert_allclose(s2["loss_before"], s1["loss_after"], rtol=1e-9)
+
+
+@pytest.mark.parametrize("n,d_in", [(256, 256), (1000, 320), (4096, 512), (777, 1160), (8192, 2048)])
+def test_hessian_tensor_core_path(n, d_in):
+    """bf16 X through the tcgen05 kernel (ragged rows and columns included) against fp64 X^T X."""
+    cfg = inputs.CONFIGS["C1"].scaled(d_in=d_in, d_out=8, n=n, seed=300 + d_in)
+    X = inputs.make_x(cfg)
+    Xd = X.cuda()
+    H = B.cdq_hessian(Xd)
+    assert B.load().cdq_last_device_status() == 0
+    Hc = H.cpu().numpy()
+    if d_in <= 1200:
+        H64, _ = oracle.hessian(X)
+        assert rel_fro(Hc, H64) <= 1e-5          # bf16 products are exact in fp32; only summation error
+    rng = np.random.default_rng(n)
+    rows = rng.integers(0, d_in, 4096); cols = rng.integers(0, d_in, 4096)
+    want = oracle.hessian_entries(X, rows, cols)
+    got = Hc[rows, cols].astype(np.float64)
+    scale = np.sqrt(oracle.hessian_entries(X, rows, rows) * oracle.hessian_entries(X, cols, cols))
+    assert np.max(np.abs(got - want) / scale) <= 1e-5
+    assert np.array_equal(Hc, Hc.T)
+    # accumulate over two row chunks == one call
+    half = (n // 2) // 8 * 8
+    H2 = B.cdq_hessian(Xd[:half])
+    H2 = B.cdq_hessian(Xd[half:], accumulate=True, out=H2)
+    assert rel_fro(H2.cpu().numpy(), Hc) <= 1e-5
