@@ -149,12 +149,16 @@ def main():
     ap.add_argument("--config", default="C1", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--d-out", type=int, default=0, help="profiling case: keep only this many output columns")
+    ap.add_argument("--n", type=int, default=0, help="profiling case: keep only this many calibration rows")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = inputs.CONFIGS[args.config]
+    if args.d_out or args.n:
+        cfg = cfg.scaled(d_out=args.d_out or cfg.d_out, n=args.n or cfg.n)
     workload = (f"{cfg.name}: d_in={cfg.d_in} d_out={cfg.d_out} n={cfg.n} X={cfg.x_dtype} W={cfg.w_dtype} "
                 f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}")
 
