@@ -72,7 +72,7 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   w.E = take(sizeof(double) * d_in * d_out);
   if (with_cd) {
     w.G = take(sizeof(double) * d_out * w.ldg);
-    w.Qt = take((size_t)d_out * d_in);
+    w.Qt = take((size_t)d_out * w.ldg);  // transposed codes, same leading dimension as G
     w.hdiag = take(sizeof(float) * w.d_pad);
     w.half_inv = take(sizeof(float) * w.d_pad);
   }
@@ -122,6 +122,10 @@ cdq_status read_device_status_after_sync() {
   if (flag == kFlagOk) return CDQ_OK;
   int zero = 0;
   cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+  if (flag == kFlagBadIndex) {
+    set_error_detail("the descent kernel produced an out-of-range coordinate and stopped");
+    return CDQ_ERR_CUDA;
+  }
   return CDQ_ERR_TIMEOUT;
 }
 
@@ -250,7 +254,7 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, G, L.ldg, col_loss, part, st));
   else CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, G, L.ldg, col_loss, st));
   CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
-  CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, Qt, st));
+  CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, d_out, Qt, L.ldg, st));
   CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (stats) {
@@ -260,13 +264,13 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   if (mode == CDQ_MODE_FAST) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
-    CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, hdiag, half_inv, steps_per_col, ctr, st));
+    CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, ctr, st));
   } else {
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
-    CDQ_CUDA(launch_cd_verify(ly, G, L.ldg, Qt, steps_per_col, ctr, st));
+    CDQ_CUDA(launch_cd_verify(ly, G, L.ldg, Qt, L.ldg, steps_per_col, ctr, st));
   }
   if (stats) CDQ_CUDA(cudaEventRecord(ev1, st));
-  CDQ_CUDA(launch_transpose_u8(Qt, d_out, d_in, Q, st));
+  CDQ_CUDA(launch_transpose_u8(Qt, d_out, d_in, L.ldg, Q, d_out, st));
   if (stats) {
     CdCounters hc;
     double lb = 0.0;

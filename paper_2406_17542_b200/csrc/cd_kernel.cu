@@ -23,14 +23,18 @@ struct CdParams {
   long long d_in, d_out;
   double* G;            // [d_out, ldg]
   long long ldg;
-  unsigned char* Qt;    // [d_out, d_in] (transposed codes)
+  unsigned char* Qt;    // [d_out, ldq] (transposed codes, ldq a multiple of 4)
+  long long ldq;
   const float* scale;   // [ng, d_out]
   const float* hdiag;   // [d_in_pad] H_ii (0 beyond d_in)
   const float* half_inv;  // [d_in_pad] 0.5 / H_ii (0 where H_ii <= 0 and beyond d_in)
   long long g, ng;
+  int ag_count;         // entries of the shared-memory scale table (>= ng)
+  unsigned gmagic;      // ceil(2^32 / g): i / g == umulhi(i, gmagic) for i, g < 2^16 (unused when g == 1)
   int L;
   long long T;
   CdCounters* ctr;
+  int* status;          // device status word
 };
 
 // ---------------------------------------------------------------------------
@@ -53,37 +57,33 @@ cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* 
   return cudaGetLastError();
 }
 
-// dst[c][r] = src[r][c] for byte matrices, 32x32 tiles through shared memory.
+// dst[c][r] = src[r][c] for byte matrices with leading dimensions, 32x32 tiles through shared memory.
 __global__ void transpose_u8_kernel(const unsigned char* __restrict__ src, long long rows, long long cols,
-                                    unsigned char* __restrict__ dst) {
+                                    long long ld_src, unsigned char* __restrict__ dst, long long ld_dst) {
   __shared__ unsigned char tile[32][33];
   const long long c0 = (long long)blockIdx.x * 32, r0 = (long long)blockIdx.y * 32;
   for (int rr = threadIdx.y; rr < 32; rr += blockDim.y) {
     const long long r = r0 + rr, c = c0 + threadIdx.x;
-    tile[rr][threadIdx.x] = (r < rows && c < cols) ? src[r * cols + c] : 0;
+    tile[rr][threadIdx.x] = (r < rows && c < cols) ? src[r * ld_src + c] : 0;
   }
   __syncthreads();
   for (int cc = threadIdx.y; cc < 32; cc += blockDim.y) {
     const long long c = c0 + cc, r = r0 + threadIdx.x;
-    if (c < cols && r < rows) dst[c * rows + r] = tile[threadIdx.x][cc];
+    if (c < cols && r < rows) dst[c * ld_dst + r] = tile[threadIdx.x][cc];
   }
 }
 
-cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols, unsigned char* dst,
-                                cudaStream_t st) {
+cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols, long long ld_src,
+                                unsigned char* dst, long long ld_dst, cudaStream_t st) {
   dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32)), block(32, 8);
-  transpose_u8_kernel<<<grid, block, 0, st>>>(src, rows, cols, dst);
+  transpose_u8_kernel<<<grid, block, 0, st>>>(src, rows, cols, ld_src, dst, ld_dst);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ unsigned order_key(float x) {
-  const unsigned u = __float_as_uint(x);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-constexpr unsigned kKeyZero = 0x80000000u;  // order_key(+0.0f)
 constexpr float kMagic = 12582912.0f;       // 1.5 * 2^23: adding it rounds to an integer
 constexpr unsigned kMagicBits = 0x4B400000u;
+constexpr unsigned kNoMove = 0xFFFFFFFFu;
 
 __device__ __forceinline__ float4 ld_row4(const float* p) {
   float4 v;
@@ -93,10 +93,23 @@ __device__ __forceinline__ float4 ld_row4(const float* p) {
   return v;
 }
 
-template <int EPT, int MAXNT, bool GROUPED>
-__global__ void __launch_bounds__(MAXNT) cd_fast_kernel(CdParams p) {
-  constexpr int NCH = EPT / 4;
-  extern __shared__ float a_s[];  // [ng] scales of the current column (GROUPED only)
+// How the scale of a coordinate is found.
+//   kPerChannel : one scale per column.  The descent runs in code units (g / a, the form of
+//                 Algorithm 1): the step 2 (r - q) is an exact small integer and the scale
+//                 drops out of every score, which saves two multiplies per coordinate.
+//   kGroupFast  : group size a multiple of 4 whose quarter divides the team size, so a thread's
+//                 chunks sit at a fixed stride in the table of group scales (shared memory).
+//   kGroupAny   : any other group size; the group of every coordinate is looked up.
+enum ScaleMode : int { kPerChannel = 0, kGroupFast = 1, kGroupAny = 2 };
+
+// One CTA ("team") owns one column at a time.  Thread t holds chunks t, t + NT, t + 2 NT, ...
+// of 4 consecutive coordinates; the gradient of the first RCH chunks lives in registers, that
+// of the other NCH - RCH chunks in shared memory (two planes of double2, conflict-free).
+// EXACT: d_in == 4 * NT * NCH, so no chunk needs a bounds test.
+template <int NCH, int RCH, int MAXNT, int MINB, int SMODE, bool EXACT>
+__global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
+  constexpr int SCH = NCH - RCH;
+  extern __shared__ __align__(16) unsigned char dyn_smem[];
   __shared__ unsigned s_key[2][32];
   __shared__ unsigned s_pk[2][32];
   __shared__ int s_col;
@@ -105,79 +118,92 @@ __global__ void __launch_bounds__(MAXNT) cd_fast_kernel(CdParams p) {
   const int lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
   const long long d_in = p.d_in;
   const int nchunks = (int)((d_in + 3) >> 2);
-  const bool vec = (d_in & 3) == 0;
-  // a 4-coordinate chunk lies inside one group unless the group size is not a multiple of 4
-  const bool chunk_scale = !GROUPED || (p.g & 3) == 0;
+  const bool vec = EXACT || (d_in & 3) == 0;
   const float topf = kMagic + (float)p.L;
+
+  auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
+  double2* gs0 = reinterpret_cast<double2*>(dyn_smem);           // [SCH][NT] coordinates 0,1 of a chunk
+  double2* gs1 = gs0 + (size_t)SCH * NT;                          // [SCH][NT] coordinates 2,3
+  float2* ag_s = reinterpret_cast<float2*>(gs1 + (size_t)SCH * NT);  // [ng] (a, 1/a), grouped modes
+  // kGroupFast: byte offset of this thread's first group entry and the stride between chunks
+  const int g4 = SMODE == kGroupFast ? (int)(p.g >> 2) : 1;
+  const float2* ag_mine = ag_s + (SMODE == kGroupFast ? tid / g4 : 0);
+  const int ag_stride = SMODE == kGroupFast ? NT / g4 : 0;
 
   unsigned long long my_committed = 0, my_converged = 0;
   double my_dsum = 0.0;
   int buf = 0;
 
   for (;;) {
-    __syncthreads();  // previous column's use of shared memory is over
+    __syncthreads();  // the previous column's use of shared memory is over
     if (tid == 0) s_col = atomicAdd(&p.ctr->next_col, 1);
     __syncthreads();
     const long long j = s_col;
     if (j >= p.d_out) break;
-#ifdef CDQ_CD_CHECKED
-    if (j < 0) { if (tid == 0) printf("cd_fast: bad column %lld\n", j); break; }
-#endif
 
     // ---- column state ----
-    double g[EPT];
-    unsigned qp[NCH];
-    float ak[GROUPED ? NCH : 1], iak[GROUPED ? NCH : 1];
-    if (GROUPED) {
-      for (long long t = tid; t < p.ng; t += NT) a_s[t] = p.scale[t * p.d_out + j];
+    float a_col = 1.f;
+    double inv_a = 1.0;
+    if (SMODE == kPerChannel) {
+      a_col = p.scale[j];
+      if (!(a_col > 0.f)) {  // constant column: its grid has one point, nothing can move
+        ++my_converged;
+        continue;
+      }
+      inv_a = 1.0 / (double)a_col;
+    } else {
+      // groups past the last real one (chunk slots beyond d_in) get a zero scale
+      for (int t = tid; t < p.ag_count; t += NT) {
+        const float a = t < p.ng ? p.scale[(long long)t * p.d_out + j] : 0.f;
+        ag_s[t] = make_float2(a, a > 0.f ? 1.0f / a : 0.f);
+      }
       __syncthreads();
     }
-    const float a_col = GROUPED ? 0.f : p.scale[j];
-    const float ia_col = (!GROUPED && a_col > 0.f) ? 1.0f / a_col : 0.f;
+    double g[RCH > 0 ? 4 * RCH : 1];
+    unsigned qp[NCH];
+    {
+      const double* gcol = p.G + j * p.ldg;
+      const unsigned char* qcol = p.Qt + j * p.ldq;
 #pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-      const int chunk = tid + NT * k;
-      const long long i0 = (long long)chunk * 4;
-      qp[k] = 0;
-#pragma unroll
-      for (int v = 0; v < 4; ++v) g[4 * k + v] = 0.0;
-      if (chunk < nchunks) {
-        if (vec) {
-          const double2 g0 = *reinterpret_cast<const double2*>(p.G + j * p.ldg + i0);
-          const double2 g1 = *reinterpret_cast<const double2*>(p.G + j * p.ldg + i0 + 2);
-          g[4 * k] = g0.x; g[4 * k + 1] = g0.y; g[4 * k + 2] = g1.x; g[4 * k + 3] = g1.y;
-          qp[k] = *reinterpret_cast<const unsigned*>(p.Qt + j * d_in + i0);
-        } else {
-#pragma unroll
-          for (int v = 0; v < 4; ++v)
-            if (i0 + v < d_in) {
-              g[4 * k + v] = p.G[j * p.ldg + i0 + v];
-              qp[k] |= (unsigned)p.Qt[j * d_in + i0 + v] << (8 * v);
-            }
+      for (int k = 0; k < NCH; ++k) {
+        const int chunk = tid + NT * k;
+        double2 g0 = make_double2(0.0, 0.0), g1 = g0;
+        qp[k] = 0;
+        if (EXACT || chunk < nchunks) {
+          g0 = *reinterpret_cast<const double2*>(gcol + (long long)chunk * 4);
+          g1 = *reinterpret_cast<const double2*>(gcol + (long long)chunk * 4 + 2);
+          qp[k] = *reinterpret_cast<const unsigned*>(qcol + (long long)chunk * 4);
         }
-      }
-      if (GROUPED) {
-        const long long gi = i0 < d_in ? i0 / p.g : 0;
-        ak[k] = a_s[gi];
-        iak[k] = ak[k] > 0.f ? 1.0f / ak[k] : 0.f;
+        if (!EXACT) {  // coordinates past d_in inside the last chunk: padding of the rows of G and Qt
+          const long long i0 = (long long)chunk * 4;
+          if (i0 + 1 >= d_in) { g0.y = 0.0; qp[k] &= 0x000000FFu; }
+          if (i0 + 2 >= d_in) { g1.x = 0.0; qp[k] &= 0x0000FFFFu; }
+          if (i0 + 3 >= d_in) { g1.y = 0.0; qp[k] &= 0x00FFFFFFu; }
+        }
+        g0.x *= inv_a; g0.y *= inv_a; g1.x *= inv_a; g1.y *= inv_a;
+        if (k < RCH) {
+          g[4 * k] = g0.x; g[4 * k + 1] = g0.y; g[4 * k + 2] = g1.x; g[4 * k + 3] = g1.y;
+        } else {
+          gs0[(k - RCH) * NT + tid] = g0;
+          gs1[(k - RCH) * NT + tid] = g1;
+        }
       }
     }
 
     // ---- descent ----
+    // The first sweep only scores: it "applies" a step of size zero along row 0.
     long long step = 0;
-    int istar = 0, dri = 0;
-    double c2 = 0.0, dd = 0.0;  // 2 d and d of the move being applied
-    bool have_move = false;
+    const float* rp = p.H;
+    double c2 = 0.0;       // twice the step being applied (code units when per-channel)
+    double col_dsum = 0.0;
     bool done = false;
     for (;;) {
-      // sweep: apply the pending move (if any) and re-score every coordinate
       float4 row[NCH];
-      const int cstar = istar >> 2, vstar = istar & 3;
-      if (have_move) {
-        const float* rp = p.H + (long long)istar * d_in;
 #pragma unroll
-        for (int k = 0; k < NCH; ++k) {
-          const int chunk = tid + NT * k;
+      for (int k = 0; k < NCH; ++k) {
+        const int chunk = tid + NT * k;
+        if (EXACT) row[k] = ld_row4(rp + (long long)chunk * 4);
+        else {
           row[k] = make_float4(0.f, 0.f, 0.f, 0.f);
           if (chunk < nchunks) {
             if (vec) row[k] = ld_row4(rp + (long long)chunk * 4);
@@ -197,154 +223,184 @@ __global__ void __launch_bounds__(MAXNT) cd_fast_kernel(CdParams p) {
         const int chunk = tid + NT * k;
         const float4 hd = __ldg(reinterpret_cast<const float4*>(p.hdiag) + chunk);
         const float4 hi = __ldg(reinterpret_cast<const float4*>(p.half_inv) + chunk);
-        float a = GROUPED ? ak[k] : a_col;
-        float ia = GROUPED ? iak[k] : ia_col;
-        const float hv[4] = {have_move ? row[k].x : 0.f, have_move ? row[k].y : 0.f,
-                             have_move ? row[k].z : 0.f, have_move ? row[k].w : 0.f};
+        float a = 1.f, ia = 1.f;
+        if (SMODE == kGroupFast) {
+          const float2 ag = ag_mine[k * ag_stride];
+          a = ag.x; ia = ag.y;
+        }
+        double gk[4];
+        if (k < RCH) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) gk[v] = g[4 * (k < RCH ? k : 0) + v];
+        } else {
+          const double2 g0 = gs0[(k - RCH) * NT + tid], g1 = gs1[(k - RCH) * NT + tid];
+          gk[0] = g0.x; gk[1] = g0.y; gk[2] = g1.x; gk[3] = g1.y;
+        }
+        const float hv[4] = {row[k].x, row[k].y, row[k].z, row[k].w};
         const float hdv[4] = {hd.x, hd.y, hd.z, hd.w};
         const float hiv[4] = {hi.x, hi.y, hi.z, hi.w};
-        if (have_move && chunk == cstar) {
-          // this thread owns the moved coordinate: exact decrease, then the new code
-#pragma unroll
-          for (int v = 0; v < 4; ++v)
-            if (v == vstar) my_dsum += dd * (dd * (double)hv[v] + g[4 * k + v]);
-          qp[k] += (unsigned)dri << (8 * vstar);
-        }
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           const int e = 4 * k + v;
-          if (GROUPED && !chunk_scale) {  // rare layout: look the scale up per coordinate
-            const long long i = (long long)chunk * 4 + v;
-            a = i < d_in ? a_s[i / p.g] : 0.f;
-            ia = a > 0.f ? 1.0f / a : 0.f;
+          if (SMODE == kGroupAny) {
+            const unsigned i = (unsigned)chunk * 4u + v;
+            const float2 ag = i < (unsigned)d_in ? ag_s[group_of(i)] : make_float2(0.f, 0.f);
+            a = ag.x; ia = ag.y;
           }
-          if (have_move) g[e] = fma(c2, (double)hv[v], g[e]);
-          const float gf = (float)g[e];
+          gk[v] = fma(c2, (double)hv[v], gk[v]);
+          const float gf = (float)gk[v];
           const float qmf = __uint_as_float(__byte_perm(qp[k], kMagicBits, 0x7650 | v));  // kMagic + q
-          float t = fmaf(-gf, ia * hiv[v], qmf);   // kMagic + rint(vertex)
+          // kMagic + rint(vertex of the coordinate's parabola), clamped to the grid
+          float t = SMODE == kPerChannel ? fmaf(-gf, hiv[v], qmf) : fmaf(-gf, ia * hiv[v], qmf);
           t = fminf(fmaxf(t, kMagic), topf);
           const float dr = t - qmf;
-          const float d = a * dr;
+          const float d = SMODE == kPerChannel ? dr : a * dr;
           const float dl = fmaf(d, hdv[v], gf) * d;
           if (dl < best) { best = dl; bpk = dr + (float)(e * 1024); }
         }
+        if (k < RCH) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) g[4 * (k < RCH ? k : 0) + v] = gk[v];
+        } else {
+          gs0[(k - RCH) * NT + tid] = make_double2(gk[0], gk[1]);
+          gs1[(k - RCH) * NT + tid] = make_double2(gk[2], gk[3]);
+        }
       }
-      if (have_move) { ++step; ++my_committed; }
       if (step >= p.T) break;
 
-      // CTA-wide argmin: (decrease, lowest coordinate, lowest level)
-      unsigned packed = 0xFFFFFFFFu;
+      // team-wide argmin: (decrease, lowest coordinate, lowest level).  `best` is negative or
+      // +0, so the complement of its bits orders the candidates; +0 becomes kNoMove.
+      unsigned packed = kNoMove;
       if (best < 0.f) {
         const int ipk = (int)bpk;
         const int e = (ipk + 512) >> 10;
         const int drq = ipk - (e << 10);
-        const int i = 4 * (tid + NT * (e >> 2)) + (e & 3);
-        packed = ((unsigned)i << 9) | (unsigned)(drq + 256);
+        // (chunk slot, thread, coordinate in chunk) orders like the coordinate index
+        packed = ((unsigned)(e >> 2) << 21) | ((unsigned)tid << 11) | ((unsigned)(e & 3) << 9) | (unsigned)(drq + 256);
       }
-      // a thread without an improving move reports exactly +0 (the compiler may have turned the
-      // running minimum into a min instruction, which can leave -0 behind)
-      unsigned key = best < 0.f ? order_key(best) : kKeyZero;
+      // (a zero step scores -0 and the compiler may keep it as the running minimum: test the sign)
+      unsigned key = best < 0.f ? ~__float_as_uint(best) : kNoMove;
       unsigned m = __reduce_min_sync(0xFFFFFFFFu, key);
-      unsigned w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : 0xFFFFFFFFu);
+      unsigned w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : kNoMove);
       if (nwarps > 1) {
         if (lane == 0) { s_key[buf][warp] = m; s_pk[buf][warp] = w; }
         __syncthreads();
-        key = lane < nwarps ? s_key[buf][lane] : 0xFFFFFFFFu;
-        packed = lane < nwarps ? s_pk[buf][lane] : 0xFFFFFFFFu;
+        key = lane < nwarps ? s_key[buf][lane] : kNoMove;
+        packed = lane < nwarps ? s_pk[buf][lane] : kNoMove;
         m = __reduce_min_sync(0xFFFFFFFFu, key);
-        w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : 0xFFFFFFFFu);
+        w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : kNoMove);
         buf ^= 1;
       }
-      if (m >= kKeyZero) { done = true; break; }  // no move lowers the loss
-      istar = (int)(w >> 9);
-      dri = (int)(w & 511u) - 256;
-#ifdef CDQ_CD_CHECKED
-      if (istar < 0 || istar >= d_in || dri == 0 || dri > p.L || dri < -p.L) {
-        if (tid == 0) printf("cd_fast: bad winner col %lld step %lld m %08x w %08x istar %d dri %d\n", j, step, m, w,
-                             istar, dri);
+      if (m == kNoMove) { done = true; break; }  // no move lowers the loss
+      const int kstar = (int)(w >> 21), tstar = (int)((w >> 11) & 1023u), vstar = (int)((w >> 9) & 3u);
+      const int dri = (int)(w & 511u) - 256;
+      const int istar = 4 * (tstar + NT * kstar) + vstar;
+      if ((unsigned)istar >= (unsigned)d_in) {  // cannot happen; never follow a bad row index
+        if (tid == 0) atomicExch(p.status, (int)kFlagBadIndex);
         break;
       }
-#endif
-      const float astar = GROUPED ? a_s[istar / p.g] : a_col;
-      dd = (double)astar * (double)dri;
-      c2 = 2.0 * dd;
-      have_move = true;
+      if (tid == tstar) {
+        const unsigned dq = (unsigned)dri << (8 * vstar);
+#pragma unroll
+        for (int k = 0; k < NCH; ++k)
+          if (k == kstar) qp[k] += dq;
+      }
+      float astar = 1.f;
+      if (SMODE != kPerChannel) astar = ag_s[group_of((unsigned)istar)].x;
+      c2 = 2.0 * ((double)astar * (double)dri);
+      rp = p.H + (long long)istar * d_in;
+      if (tid == 0) col_dsum += (double)__uint_as_float(~m);
+      ++step;
     }
     if (done) ++my_converged;
+    my_committed += (unsigned long long)step;
+    my_dsum += SMODE == kPerChannel ? col_dsum * ((double)a_col * (double)a_col) : col_dsum;
 
     // ---- write the codes back ----
+    {
+      unsigned char* qcol = p.Qt + j * p.ldq;
 #pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-      const int chunk = tid + NT * k;
-      const long long i0 = (long long)chunk * 4;
-      if (chunk < nchunks) {
-        if (vec) *reinterpret_cast<unsigned*>(p.Qt + j * d_in + i0) = qp[k];
-        else {
-#pragma unroll
-          for (int v = 0; v < 4; ++v)
-            if (i0 + v < d_in) p.Qt[j * d_in + i0 + v] = (unsigned char)(qp[k] >> (8 * v));
-        }
+      for (int k = 0; k < NCH; ++k) {
+        const int chunk = tid + NT * k;
+        if (EXACT || chunk < nchunks) *reinterpret_cast<unsigned*>(qcol + (long long)chunk * 4) = qp[k];
       }
     }
   }
 
   // ---- statistics ----
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) my_dsum += __shfl_xor_sync(0xFFFFFFFFu, my_dsum, o);
-  if (lane == 0 && my_dsum != 0.0) atomicAdd(&p.ctr->delta_sum, my_dsum);
   if (tid == 0) {
+    if (my_dsum != 0.0) atomicAdd(&p.ctr->delta_sum, my_dsum);
     if (my_committed) atomicAdd(&p.ctr->committed, my_committed);
     if (my_converged) atomicAdd(&p.ctr->converged, my_converged);
   }
 }
 
-template <int EPT, int MAXNT>
-static cudaError_t launch_cd_fast_t(const CdParams& p, int nt, bool grouped, cudaStream_t st) {
+template <int NCH, int RCH, int MAXNT, int MINB, int SMODE, bool EXACT>
+static cudaError_t launch_cd_cfg(CdParams p, int nt, cudaStream_t st) {
+  p.ag_count = (int)p.ng;
+  if (SMODE == kGroupFast) {
+    const int g4 = (int)(p.g >> 2), slots = (nt * NCH + g4 - 1) / g4;
+    if (slots > p.ag_count) p.ag_count = slots;
+  }
+  auto kern = cd_fast_kernel<NCH, RCH, MAXNT, MINB, SMODE, EXACT>;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const size_t smem = grouped ? sizeof(float) * (size_t)p.ng : 0;
-  int per_sm = 1;
+  const size_t smem = (size_t)(NCH - RCH) * nt * 2 * sizeof(double2) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
   cudaError_t e;
-  if (grouped) {
-    if (smem > 48 * 1024) {
-      e = cudaFuncSetAttribute(cd_fast_kernel<EPT, MAXNT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-    }
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cd_fast_kernel<EPT, MAXNT, true>, nt, smem);
-  } else {
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cd_fast_kernel<EPT, MAXNT, false>, nt, smem);
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
   }
+  int per_sm = 1;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, nt, smem);
   if (e != cudaSuccess) return e;
-  if (per_sm < 1) per_sm = 1;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
   long long blocks = (long long)sms * per_sm;
   if (blocks > p.d_out) blocks = p.d_out;
-  if (grouped) cd_fast_kernel<EPT, MAXNT, true><<<(unsigned)blocks, nt, smem, st>>>(p);
-  else cd_fast_kernel<EPT, MAXNT, false><<<(unsigned)blocks, nt, smem, st>>>(p);
+  kern<<<(unsigned)blocks, nt, smem, st>>>(p);
   return cudaGetLastError();
 }
 
+// Picks the scale mode and whether the team covers d_in exactly.
+template <int NCH, int RCH, int MAXNT, int MINB>
+static cudaError_t launch_cd_shape(const CdParams& p, int nt, cudaStream_t st) {
+  const bool exact = p.d_in == 4ll * nt * NCH;
+  int smode = kPerChannel;
+  if (p.ng > 1) smode = ((p.g & 3) == 0 && nt % (int)(p.g >> 2) == 0) ? kGroupFast : kGroupAny;
+  if (smode == kPerChannel)
+    return exact ? launch_cd_cfg<NCH, RCH, MAXNT, MINB, kPerChannel, true>(p, nt, st)
+                 : launch_cd_cfg<NCH, RCH, MAXNT, MINB, kPerChannel, false>(p, nt, st);
+  if (smode == kGroupFast)
+    return exact ? launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupFast, true>(p, nt, st)
+                 : launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupFast, false>(p, nt, st);
+  return launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupAny, false>(p, nt, st);
+}
+
 long long cd_fast_pad(long long d_in) {
-  // hdiag / half_inv are read in 16-byte pieces by every thread slot of a team, so they are
-  // padded to beyond the largest team footprint (threads are a multiple of 32, 32 slots each).
+  // hdiag / half_inv are read in 16-byte pieces by every chunk slot of a team, so they are
+  // padded to beyond the largest team footprint (at most 32 extra threads of 32 coordinates).
   return (d_in + 2048 + 255) / 256 * 256;
 }
 
 bool cd_fast_supported(long long d_in) { return d_in >= 1 && d_in <= 18432; }
 
-cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, const float* hdiag,
-                           const float* half_inv, long long steps_per_col, CdCounters* ctr, cudaStream_t st) {
+cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
+                           const float* hdiag, const float* half_inv, long long steps_per_col, CdCounters* ctr,
+                           cudaStream_t st) {
   CdParams p{};
-  p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.scale = ly.scale;
+  p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
   p.hdiag = hdiag; p.half_inv = half_inv; p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
-  const bool grouped = ly.ng > 1;
+  p.status = device_status_word();
+  if (!p.status) return cudaErrorInvalidSymbol;
+  p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
   const long long d = ly.d_in;
   auto team = [&](int ept) { return (int)(((d + ept - 1) / ept + 31) / 32 * 32); };
-  if (d <= 512) return launch_cd_fast_t<8, 64>(p, team(8), grouped, st);
-  if (d <= 4096) return launch_cd_fast_t<16, 256>(p, team(16), grouped, st);
-  if (d <= 8192) return launch_cd_fast_t<32, 256>(p, team(32), grouped, st);
-  if (d <= 14336) return launch_cd_fast_t<32, 448>(p, team(32), grouped, st);
-  return launch_cd_fast_t<32, 576>(p, team(32), grouped, st);
+  if (d <= 512) return launch_cd_shape<2, 2, 64, 8>(p, team(8), st);
+  if (d <= 4096) return launch_cd_shape<4, 4, 256, 3>(p, team(16), st);
+  if (d <= 8192) return launch_cd_shape<8, 8, 256, 2>(p, team(32), st);
+  if (d <= 14336) return launch_cd_shape<8, 8, 448, 1>(p, team(32), st);
+  return launch_cd_shape<8, 6, 576, 1>(p, team(32), st);
 }
 
 // ---------------------------------------------------------------------------
@@ -359,7 +415,7 @@ __global__ void __launch_bounds__(128) cd_verify_kernel(CdParams p) {
   const int tid = threadIdx.x;
   const long long d_in = p.d_in;
   double* g = p.G + j * p.ldg;
-  unsigned char* q = p.Qt + j * d_in;
+  unsigned char* q = p.Qt + j * p.ldq;
   unsigned long long moves = 0;
   double dsum = 0.0;
   bool done = false;
@@ -411,10 +467,10 @@ __global__ void __launch_bounds__(128) cd_verify_kernel(CdParams p) {
   }
 }
 
-cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long steps_per_col,
-                             CdCounters* ctr, cudaStream_t st) {
+cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
+                             long long steps_per_col, CdCounters* ctr, cudaStream_t st) {
   CdParams p{};
-  p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.scale = ly.scale;
+  p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
   p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
   cd_verify_kernel<<<(unsigned)ly.d_out, 128, 0, st>>>(p);
   return cudaGetLastError();

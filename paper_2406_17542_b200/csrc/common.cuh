@@ -15,7 +15,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 // Device status word: kernels with bounded waits record a failure here.
-enum DeviceFlag : int { kFlagOk = 0, kFlagWaitTimeout = 1 };
+enum DeviceFlag : int { kFlagOk = 0, kFlagWaitTimeout = 1, kFlagBadIndex = 2 };
 int* device_status_word();  // device address of the status word (per process)
 
 // Text returned by cdq_last_error_detail().
@@ -89,16 +89,16 @@ struct CdCounters {            // lives in the workspace, zeroed by the launcher
   int next_col;
   int pad;
 };
-cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols,
-                                unsigned char* dst, cudaStream_t st);  // dst[c][r] = src[r][c]
+cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols, long long ld_src,
+                                unsigned char* dst, long long ld_dst, cudaStream_t st);  // dst[c][r] = src[r][c]
 long long cd_fast_pad(long long d_in);      // padded length of hdiag / half_inv
 bool cd_fast_supported(long long d_in);
 cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* half_inv,
                         cudaStream_t st);
-cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt,
+cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                            const float* hdiag, const float* half_inv, long long steps_per_col,
                            CdCounters* ctr, cudaStream_t st);
-cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt,
+cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                              long long steps_per_col, CdCounters* ctr, cudaStream_t st);
 cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st);  // ascending order
 
