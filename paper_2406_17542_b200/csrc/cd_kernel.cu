@@ -13,29 +13,13 @@
 //   r = clamp(rint(q_i - g_i / (2 a_i H_ii)), 0, L),
 // so the level scan of Algorithm 1 line 5 costs O(1) per coordinate.
 #include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
+#include "cd_params.cuh"
 
 namespace cdq {
 
-struct CdParams {
-  const float* H;
-  long long d_in, d_out;
-  double* G;            // [d_out, ldg]
-  long long ldg;
-  unsigned char* Qt;    // [d_out, ldq] (transposed codes, ldq a multiple of 4)
-  long long ldq;
-  const float* scale;   // [ng, d_out]
-  const float* hdiag;   // [d_in_pad] H_ii (0 beyond d_in)
-  const float* half_inv;  // [d_in_pad] 0.5 / H_ii (0 where H_ii <= 0 and beyond d_in)
-  long long g, ng;
-  int ag_count;         // entries of the shared-memory scale table (>= ng)
-  unsigned gmagic;      // ceil(2^32 / g): i / g == umulhi(i, gmagic) for i, g < 2^16 (unused when g == 1)
-  int L;
-  long long T;
-  CdCounters* ctr;
-  int* status;          // device status word
-};
 
 // ---------------------------------------------------------------------------
 __global__ void diag_kernel(const float* __restrict__ H, long long d_in, long long d_pad,
@@ -81,10 +65,6 @@ cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long l
 }
 
 // ---------------------------------------------------------------------------
-constexpr float kMagic = 12582912.0f;       // 1.5 * 2^23: adding it rounds to an integer
-constexpr unsigned kMagicBits = 0x4B400000u;
-constexpr unsigned kNoMove = 0xFFFFFFFFu;
-
 __device__ __forceinline__ float4 ld_row4(const float* p) {
   float4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
@@ -92,15 +72,6 @@ __device__ __forceinline__ float4 ld_row4(const float* p) {
                : "l"(p));
   return v;
 }
-
-// How the scale of a coordinate is found.
-//   kPerChannel : one scale per column.  The descent runs in code units (g / a, the form of
-//                 Algorithm 1): the step 2 (r - q) is an exact small integer and the scale
-//                 drops out of every score, which saves two multiplies per coordinate.
-//   kGroupFast  : group size a multiple of 4 whose quarter divides the team size, so a thread's
-//                 chunks sit at a fixed stride in the table of group scales (shared memory).
-//   kGroupAny   : any other group size; the group of every coordinate is looked up.
-enum ScaleMode : int { kPerChannel = 0, kGroupFast = 1, kGroupAny = 2 };
 
 // One CTA ("team") owns one column at a time.  Thread t holds chunks t, t + NT, t + 2 NT, ...
 // of 4 consecutive coordinates; the gradient of the first RCH chunks lives in registers, that
@@ -394,6 +365,12 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
   p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
+  // CDQ_CD_KERNEL=plain in the environment keeps the rows in registers (no bulk copies, no clusters)
+  static const bool force_plain = [] { const char* e = getenv("CDQ_CD_KERNEL"); return e && e[0] == 'p'; }();
+  if (!force_plain) {
+    const cudaError_t e = launch_cd_tma(p, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
   const long long d = ly.d_in;
   auto team = [&](int ept) { return (int)(((d + ept - 1) / ept + 31) / 32 * 32); };
   if (d <= 512) return launch_cd_shape<2, 2, 64, 8>(p, team(8), st);
