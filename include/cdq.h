@@ -81,7 +81,8 @@ typedef struct {
   unsigned long long committed;         /* moves actually made                           */
   unsigned long long columns_converged; /* columns that ran out of improving moves       */
   double loss_before;                   /* sum_j e_j^T H e_j at entry (from G0)          */
-  double loss_after;                    /* loss_before + sum of committed decreases      */
+  double loss_after;                    /* loss_before + sum of committed decreases (FAST:
+                                           the fp32 scores of the moves, ~1e-7 relative)  */
   double kernel_ms;                     /* device time of the descent kernel alone (CUDA
                                            events on `stream`), for roofline accounting   */
 } cdq_cd_stats;

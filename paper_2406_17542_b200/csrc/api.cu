@@ -78,7 +78,7 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   }
   w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
   w.col_loss = take(sizeof(double) * d_out);
-  w.scalars = take(256);  // [0]: double loss sum; [64..): CdCounters
+  w.scalars = take(256);  // [0]: loss sum; [64..): CdCounters
   w.total = off;
   return w;
 }
@@ -231,7 +231,6 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);
   if (s != CDQ_OK) return s;
-  if (mode == CDQ_MODE_FAST && !cd_fast_supported(d_in)) return CDQ_ERR_UNSUPPORTED;
   const SolveWs L = solve_ws_layout(d_in, d_out, mode, true);
   s = check_ws(ws, ws_bytes, L.total);
   if (s != CDQ_OK) return s;
@@ -261,7 +260,10 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
     CDQ_CUDA(cudaEventCreate(&ev0));
     CDQ_CUDA(cudaEventCreate(&ev1));
   }
-  if (mode == CDQ_MODE_FAST) {
+  // shapes the fast kernels do not cover (a group size that is not a multiple of 4, very long
+  // columns) take the fixed-order fp64 kernel: slower, same result
+  const bool fast_cd = mode == CDQ_MODE_FAST && cd_fast_supported(d_in, ly.g);
+  if (fast_cd) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
     CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, ctr, st));

@@ -17,27 +17,30 @@
 
 #include "common.cuh"
 #include "cd_params.cuh"
+#include "cd_sweep.cuh"
 
 namespace cdq {
 
 
 // ---------------------------------------------------------------------------
+// Diagonal of H for the scoring arithmetic: hdiag = H_ii, hs = 0.5 / H_ii (0 for a dead feature
+// and in the padding beyond d_in).
 __global__ void diag_kernel(const float* __restrict__ H, long long d_in, long long d_pad,
-                            float* __restrict__ hdiag, float* __restrict__ half_inv) {
+                            float* __restrict__ hdiag, float* __restrict__ hs) {
   const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (i >= d_pad) return;
-  float h = 0.f, hi = 0.f;
+  float h = 0.f, w = 0.f;
   if (i < d_in) {
     h = H[i * d_in + i];
-    hi = h > 0.f ? 0.5f / h : 0.f;
+    if (!(h > 0.f)) h = 0.f;
+    w = h > 0.f ? 0.5f / h : 0.f;
   }
   hdiag[i] = h;
-  half_inv[i] = hi;
+  hs[i] = w;
 }
 
-cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* half_inv,
-                        cudaStream_t st) {
-  diag_kernel<<<(unsigned)((d_pad + 255) / 256), 256, 0, st>>>(H, d_in, d_pad, hdiag, half_inv);
+cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* hs, cudaStream_t st) {
+  diag_kernel<<<(unsigned)((d_pad + 255) / 256), 256, 0, st>>>(H, d_in, d_pad, hdiag, hs);
   return cudaGetLastError();
 }
 
@@ -74,15 +77,12 @@ __device__ __forceinline__ float4 ld_row4(const float* p) {
 }
 
 // One CTA ("team") owns one column at a time.  Thread t holds chunks t, t + NT, t + 2 NT, ...
-// of 4 consecutive coordinates; the gradient of the first RCH chunks lives in registers, that
-// of the other NCH - RCH chunks in shared memory (two planes of double2, conflict-free).
+// of 4 consecutive coordinates: gradient (fp64) and codes (packed bytes) in registers.
 // EXACT: d_in == 4 * NT * NCH, so no chunk needs a bounds test.
-template <int NCH, int RCH, int MAXNT, int MINB, int SMODE, bool EXACT>
+template <int NCH, int MAXNT, int MINB, int SMODE, bool EXACT>
 __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
-  constexpr int SCH = NCH - RCH;
   extern __shared__ __align__(16) unsigned char dyn_smem[];
-  __shared__ unsigned s_key[2][32];
-  __shared__ unsigned s_pk[2][32];
+  __shared__ __align__(8) uint2 s_exch[2][32];
   __shared__ int s_col;
 
   const int tid = threadIdx.x, NT = blockDim.x;
@@ -90,20 +90,28 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
   const long long d_in = p.d_in;
   const int nchunks = (int)((d_in + 3) >> 2);
   const bool vec = EXACT || (d_in & 3) == 0;
-  const float topf = kMagic + (float)p.L;
+  const float top = kMagic + (float)p.L;
 
   auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
-  double2* gs0 = reinterpret_cast<double2*>(dyn_smem);           // [SCH][NT] coordinates 0,1 of a chunk
-  double2* gs1 = gs0 + (size_t)SCH * NT;                          // [SCH][NT] coordinates 2,3
-  float2* ag_s = reinterpret_cast<float2*>(gs1 + (size_t)SCH * NT);  // [ng] (a, 1/a), grouped modes
-  // kGroupFast: byte offset of this thread's first group entry and the stride between chunks
+  float2* ag_s = reinterpret_cast<float2*>(dyn_smem);  // [ag_count] (a, 1/a), grouped modes
   const int g4 = SMODE == kGroupFast ? (int)(p.g >> 2) : 1;
   const float2* ag_mine = ag_s + (SMODE == kGroupFast ? tid / g4 : 0);
   const int ag_stride = SMODE == kGroupFast ? NT / g4 : 0;
+  // scale (a, 1/a) of chunk slot k of this thread; kGroupAny keeps one scale per chunk only when
+  // the group size is a multiple of 4, otherwise the launcher does not pick this kernel
+  auto chunk_scale = [&](int k, float& a, float& ia) {
+    a = 1.f; ia = 1.f;
+    if (SMODE == kGroupFast) { const float2 ag = ag_mine[k * ag_stride]; a = ag.x; ia = ag.y; }
+    if (SMODE == kGroupAny) {
+      const unsigned i = (unsigned)(tid + NT * k) * 4u;
+      const float2 ag = i < (unsigned)d_in ? ag_s[group_of(i)] : make_float2(0.f, 0.f);
+      a = ag.x; ia = ag.y;
+    }
+  };
 
   unsigned long long my_committed = 0, my_converged = 0;
   double my_dsum = 0.0;
-  int buf = 0;
+  int xbuf = 0;
 
   for (;;) {
     __syncthreads();  // the previous column's use of shared memory is over
@@ -114,14 +122,14 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
 
     // ---- column state ----
     float a_col = 1.f;
-    double inv_a = 1.0;
+    double gscale = 1.0;   // what the stored gradient is multiplied by on load
     if (SMODE == kPerChannel) {
       a_col = p.scale[j];
       if (!(a_col > 0.f)) {  // constant column: its grid has one point, nothing can move
-        ++my_converged;
+        if (tid == 0) ++my_converged;
         continue;
       }
-      inv_a = 1.0 / (double)a_col;
+      gscale = 1.0 / (double)a_col;
     } else {
       // groups past the last real one (chunk slots beyond d_in) get a zero scale
       for (int t = tid; t < p.ag_count; t += NT) {
@@ -130,7 +138,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
       }
       __syncthreads();
     }
-    double g[RCH > 0 ? 4 * RCH : 1];
+    double g[4 * NCH];
     unsigned qp[NCH];
     {
       const double* gcol = p.G + j * p.ldg;
@@ -151,13 +159,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
           if (i0 + 2 >= d_in) { g1.x = 0.0; qp[k] &= 0x0000FFFFu; }
           if (i0 + 3 >= d_in) { g1.y = 0.0; qp[k] &= 0x00FFFFFFu; }
         }
-        g0.x *= inv_a; g0.y *= inv_a; g1.x *= inv_a; g1.y *= inv_a;
-        if (k < RCH) {
-          g[4 * k] = g0.x; g[4 * k + 1] = g0.y; g[4 * k + 2] = g1.x; g[4 * k + 3] = g1.y;
-        } else {
-          gs0[(k - RCH) * NT + tid] = g0;
-          gs1[(k - RCH) * NT + tid] = g1;
-        }
+        g[4 * k] = g0.x * gscale; g[4 * k + 1] = g0.y * gscale; g[4 * k + 2] = g1.x * gscale; g[4 * k + 3] = g1.y * gscale;
       }
     }
 
@@ -188,79 +190,35 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
           }
         }
       }
-      float best = 0.f, bpk = 0.f;
+      SweepBest sb;
+      sb.init();
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         const int chunk = tid + NT * k;
         const float4 hd = __ldg(reinterpret_cast<const float4*>(p.hdiag) + chunk);
-        const float4 hi = __ldg(reinterpret_cast<const float4*>(p.half_inv) + chunk);
-        float a = 1.f, ia = 1.f;
-        if (SMODE == kGroupFast) {
-          const float2 ag = ag_mine[k * ag_stride];
-          a = ag.x; ia = ag.y;
-        }
-        double gk[4];
-        if (k < RCH) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) gk[v] = g[4 * (k < RCH ? k : 0) + v];
-        } else {
-          const double2 g0 = gs0[(k - RCH) * NT + tid], g1 = gs1[(k - RCH) * NT + tid];
-          gk[0] = g0.x; gk[1] = g0.y; gk[2] = g1.x; gk[3] = g1.y;
-        }
-        const float hv[4] = {row[k].x, row[k].y, row[k].z, row[k].w};
-        const float hdv[4] = {hd.x, hd.y, hd.z, hd.w};
-        const float hiv[4] = {hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const int e = 4 * k + v;
-          if (SMODE == kGroupAny) {
-            const unsigned i = (unsigned)chunk * 4u + v;
-            const float2 ag = i < (unsigned)d_in ? ag_s[group_of(i)] : make_float2(0.f, 0.f);
-            a = ag.x; ia = ag.y;
-          }
-          gk[v] = fma(c2, (double)hv[v], gk[v]);
-          const float gf = (float)gk[v];
-          const float qmf = __uint_as_float(__byte_perm(qp[k], kMagicBits, 0x7650 | v));  // kMagic + q
-          // kMagic + rint(vertex of the coordinate's parabola), clamped to the grid
-          float t = SMODE == kPerChannel ? fmaf(-gf, hiv[v], qmf) : fmaf(-gf, ia * hiv[v], qmf);
-          t = fminf(fmaxf(t, kMagic), topf);
-          const float dr = t - qmf;
-          const float d = SMODE == kPerChannel ? dr : a * dr;
-          const float dl = fmaf(d, hdv[v], gf) * d;
-          if (dl < best) { best = dl; bpk = dr + (float)(e * 1024); }
-        }
-        if (k < RCH) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) g[4 * (k < RCH ? k : 0) + v] = gk[v];
-        } else {
-          gs0[(k - RCH) * NT + tid] = make_double2(gk[0], gk[1]);
-          gs1[(k - RCH) * NT + tid] = make_double2(gk[2], gk[3]);
-        }
+        const float4 hs = __ldg(reinterpret_cast<const float4*>(p.hs) + chunk);
+        float a, ia;
+        chunk_scale(k, a, ia);
+        double gk[4] = {g[4 * k], g[4 * k + 1], g[4 * k + 2], g[4 * k + 3]};
+        sweep_chunk<SMODE>(gk, row[k], hd, hs, qp[k], c2, a, ia, top, k, sb);
+        g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
       }
       if (step >= p.T) break;
 
-      // team-wide argmin: (decrease, lowest coordinate, lowest level).  `best` is negative or
-      // +0, so the complement of its bits orders the candidates; +0 becomes kNoMove.
-      unsigned packed = kNoMove;
-      if (best < 0.f) {
-        const int ipk = (int)bpk;
-        const int e = (ipk + 512) >> 10;
-        const int drq = ipk - (e << 10);
-        // (chunk slot, thread, coordinate in chunk) orders like the coordinate index
-        packed = ((unsigned)(e >> 2) << 21) | ((unsigned)tid << 11) | ((unsigned)(e & 3) << 9) | (unsigned)(drq + 256);
-      }
-      // (a zero step scores -0 and the compiler may keep it as the running minimum: test the sign)
-      unsigned key = best < 0.f ? ~__float_as_uint(best) : kNoMove;
+      // ---- team-wide argmin: (decrease, lowest coordinate, lowest level) ----
+      unsigned key, packed;
+      sweep_candidate(sb, tid, key, packed);
       unsigned m = __reduce_min_sync(0xFFFFFFFFu, key);
       unsigned w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : kNoMove);
       if (nwarps > 1) {
-        if (lane == 0) { s_key[buf][warp] = m; s_pk[buf][warp] = w; }
+        if (lane == 0) s_exch[xbuf][warp] = make_uint2(m, w);
         __syncthreads();
-        key = lane < nwarps ? s_key[buf][lane] : kNoMove;
-        packed = lane < nwarps ? s_pk[buf][lane] : kNoMove;
-        m = __reduce_min_sync(0xFFFFFFFFu, key);
-        w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : kNoMove);
-        buf ^= 1;
+        const uint2 x = lane < nwarps ? s_exch[xbuf][lane] : make_uint2(kNoMove, kNoMove);
+        m = __reduce_min_sync(0xFFFFFFFFu, x.x);
+        w = __reduce_min_sync(0xFFFFFFFFu, x.x == m ? x.y : kNoMove);
+        xbuf ^= 1;
+      } else {
+        __syncwarp();
       }
       if (m == kNoMove) { done = true; break; }  // no move lowers the loss
       const int kstar = (int)(w >> 21), tstar = (int)((w >> 11) & 1023u), vstar = (int)((w >> 9) & 3u);
@@ -283,9 +241,11 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
       ++step;
     }
-    if (done) ++my_converged;
-    my_committed += (unsigned long long)step;
-    my_dsum += SMODE == kPerChannel ? col_dsum * ((double)a_col * (double)a_col) : col_dsum;
+    if (tid == 0) {
+      if (done) ++my_converged;
+      my_committed += (unsigned long long)step;
+      my_dsum += SMODE == kPerChannel ? col_dsum * ((double)a_col * (double)a_col) : col_dsum;
+    }
 
     // ---- write the codes back ----
     {
@@ -306,18 +266,18 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
   }
 }
 
-template <int NCH, int RCH, int MAXNT, int MINB, int SMODE, bool EXACT>
+template <int NCH, int MAXNT, int MINB, int SMODE, bool EXACT>
 static cudaError_t launch_cd_cfg(CdParams p, int nt, cudaStream_t st) {
   p.ag_count = (int)p.ng;
   if (SMODE == kGroupFast) {
     const int g4 = (int)(p.g >> 2), slots = (nt * NCH + g4 - 1) / g4;
     if (slots > p.ag_count) p.ag_count = slots;
   }
-  auto kern = cd_fast_kernel<NCH, RCH, MAXNT, MINB, SMODE, EXACT>;
+  auto kern = cd_fast_kernel<NCH, MAXNT, MINB, SMODE, EXACT>;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const size_t smem = (size_t)(NCH - RCH) * nt * 2 * sizeof(double2) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
+  const size_t smem = SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count;
   cudaError_t e;
   if (smem > 48 * 1024) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -334,18 +294,18 @@ static cudaError_t launch_cd_cfg(CdParams p, int nt, cudaStream_t st) {
 }
 
 // Picks the scale mode and whether the team covers d_in exactly.
-template <int NCH, int RCH, int MAXNT, int MINB>
+template <int NCH, int MAXNT, int MINB>
 static cudaError_t launch_cd_shape(const CdParams& p, int nt, cudaStream_t st) {
   const bool exact = p.d_in == 4ll * nt * NCH;
-  int smode = kPerChannel;
-  if (p.ng > 1) smode = ((p.g & 3) == 0 && nt % (int)(p.g >> 2) == 0) ? kGroupFast : kGroupAny;
+  const int smode = cd_scale_mode(p, nt);
+  if (smode < 0) return cudaErrorNotSupported;
   if (smode == kPerChannel)
-    return exact ? launch_cd_cfg<NCH, RCH, MAXNT, MINB, kPerChannel, true>(p, nt, st)
-                 : launch_cd_cfg<NCH, RCH, MAXNT, MINB, kPerChannel, false>(p, nt, st);
+    return exact ? launch_cd_cfg<NCH, MAXNT, MINB, kPerChannel, true>(p, nt, st)
+                 : launch_cd_cfg<NCH, MAXNT, MINB, kPerChannel, false>(p, nt, st);
   if (smode == kGroupFast)
-    return exact ? launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupFast, true>(p, nt, st)
-                 : launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupFast, false>(p, nt, st);
-  return launch_cd_cfg<NCH, RCH, MAXNT, MINB, kGroupAny, false>(p, nt, st);
+    return exact ? launch_cd_cfg<NCH, MAXNT, MINB, kGroupFast, true>(p, nt, st)
+                 : launch_cd_cfg<NCH, MAXNT, MINB, kGroupFast, false>(p, nt, st);
+  return launch_cd_cfg<NCH, MAXNT, MINB, kGroupAny, false>(p, nt, st);
 }
 
 long long cd_fast_pad(long long d_in) {
@@ -354,30 +314,40 @@ long long cd_fast_pad(long long d_in) {
   return (d_in + 2048 + 255) / 256 * 256;
 }
 
-bool cd_fast_supported(long long d_in) { return d_in >= 1 && d_in <= 18432; }
+// The fast kernels keep one scale per chunk of 4 coordinates, so grouped grids need a group
+// size that is a multiple of 4 (any group size runs in the verification mode).
+bool cd_fast_supported(long long d_in, long long g) {
+  return d_in >= 1 && d_in <= 18432 && (g == d_in || (g & 3) == 0);
+}
 
 cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
-                           const float* hdiag, const float* half_inv, long long steps_per_col, CdCounters* ctr,
-                           cudaStream_t st) {
+                           const float* hdiag, const float* hs, long long steps_per_col,
+                           CdCounters* ctr, cudaStream_t st) {
   CdParams p{};
   p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
-  p.hdiag = hdiag; p.half_inv = half_inv; p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
+  p.hdiag = hdiag; p.hs = hs; p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
   p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
-  // CDQ_CD_KERNEL=plain in the environment keeps the rows in registers (no bulk copies, no clusters)
-  static const bool force_plain = [] { const char* e = getenv("CDQ_CD_KERNEL"); return e && e[0] == 'p'; }();
-  if (!force_plain) {
+  // CDQ_CD_KERNEL=plain in the environment keeps the rows in registers (no bulk copies);
+  // CDQ_CD_KERNEL=tma stages them through shared memory whenever the shape allows
+  static const int force = [] {
+    const char* e = getenv("CDQ_CD_KERNEL");
+    return !e ? 0 : (e[0] == 'p' ? 1 : (e[0] == 't' ? 2 : 0));
+  }();
+  const long long d = ly.d_in;
+  // rows that come out of L2 (H up to 64 MB) are quickest as plain loads; larger ones as bulk copies
+  const bool want_tma = force == 2 || (force == 0 && d > 4096);
+  if (want_tma) {
     const cudaError_t e = launch_cd_tma(p, st);
     if (e != cudaErrorNotSupported) return e;
   }
-  const long long d = ly.d_in;
   auto team = [&](int ept) { return (int)(((d + ept - 1) / ept + 31) / 32 * 32); };
-  if (d <= 512) return launch_cd_shape<2, 2, 64, 8>(p, team(8), st);
-  if (d <= 4096) return launch_cd_shape<4, 4, 256, 3>(p, team(16), st);
-  if (d <= 8192) return launch_cd_shape<8, 8, 256, 2>(p, team(32), st);
-  if (d <= 14336) return launch_cd_shape<8, 8, 448, 1>(p, team(32), st);
-  return launch_cd_shape<8, 6, 576, 1>(p, team(32), st);
+  if (d <= 512) return launch_cd_shape<2, 64, 8>(p, team(8), st);
+  if (d <= 4096) return launch_cd_shape<4, 256, 3>(p, team(16), st);
+  if (d <= 8192) return launch_cd_shape<8, 256, 2>(p, team(32), st);
+  if (d <= 14336) return launch_cd_shape<8, 448, 1>(p, team(32), st);
+  return launch_cd_shape<8, 576, 1>(p, team(32), st);
 }
 
 // ---------------------------------------------------------------------------

@@ -14,7 +14,7 @@ struct CdParams {
   long long ldq;
   const float* scale;   // [ng, d_out]
   const float* hdiag;   // [d_in_pad] H_ii (0 beyond d_in)
-  const float* half_inv;  // [d_in_pad] 0.5 / H_ii (0 where H_ii <= 0 and beyond d_in)
+  const float* hs;      // [d_in_pad] 0.5 / H_ii (0 where H_ii <= 0 and beyond d_in)
   long long g, ng;
   int ag_count;         // entries of the shared-memory scale table (>= ng)
   unsigned gmagic;      // ceil(2^32 / g): i / g == umulhi(i, gmagic) for i, g < 2^16 (unused when g == 1)
@@ -37,9 +37,16 @@ constexpr unsigned kNoMove = 0xFFFFFFFFu;
 //   kGroupAny   : any other group size; the group of every coordinate is looked up.
 enum ScaleMode : int { kPerChannel = 0, kGroupFast = 1, kGroupAny = 2 };
 
-// cd_kernel_tma.cu: rows staged through shared memory by bulk copies, column optionally split
-// over a thread-block cluster.  Returns cudaErrorNotSupported when the shape has no such
-// configuration (the caller then uses the plain kernel).
+// Scale mode of a layer for a team of nt threads (-1: no fast kernel handles it).
+inline int cd_scale_mode(const CdParams& p, int nt) {
+  if (p.ng <= 1) return kPerChannel;
+  if (p.g & 3) return -1;
+  return nt % (int)(p.g >> 2) == 0 ? kGroupFast : kGroupAny;
+}
+
+// cd_kernel_tma.cu: rows staged through shared memory by bulk copies.  Returns
+// cudaErrorNotSupported when the shape has no such configuration (the caller then uses the
+// plain kernel).
 cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st);
 
 }  // namespace cdq

@@ -91,12 +91,12 @@ struct CdCounters {            // lives in the workspace, zeroed by the launcher
 };
 cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols, long long ld_src,
                                 unsigned char* dst, long long ld_dst, cudaStream_t st);  // dst[c][r] = src[r][c]
-long long cd_fast_pad(long long d_in);      // padded length of hdiag / half_inv
-bool cd_fast_supported(long long d_in);
-cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* half_inv,
-                        cudaStream_t st);
+long long cd_fast_pad(long long d_in);      // padded length of hdiag / hs
+bool cd_fast_supported(long long d_in, long long g);
+// hdiag = H_ii, hs = 0.5 / H_ii
+cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* hs, cudaStream_t st);
 cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
-                           const float* hdiag, const float* half_inv, long long steps_per_col,
+                           const float* hdiag, const float* hs, long long steps_per_col,
                            CdCounters* ctr, cudaStream_t st);
 cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                              long long steps_per_col, CdCounters* ctr, cudaStream_t st);

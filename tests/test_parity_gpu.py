@@ -137,7 +137,8 @@ def test_resume_from_previous_codes():
     s1 = B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, 1)
     s2 = B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, 1)
     assert s2["committed"] == 0 and s2["columns_converged"] == cfg.d_out
-    np.testing.assert_allclose(s2["loss_before"], s1["loss_after"], rtol=1e-9)
+    # loss_after adds up the committed decreases, which the production mode scores in fp32
+    np.testing.assert_allclose(s2["loss_before"], s1["loss_after"], rtol=1e-6)
 
 
 @pytest.mark.parametrize("n,d_in", [(256, 256), (1000, 320), (4096, 512), (777, 1160), (8192, 2048)])
