@@ -42,6 +42,7 @@ struct Params {
   long long n, d_in;
   int tiles_m, ntiles, splits, kblocks;
   float* partials;   // [splits][ntiles][BM*BN]
+  const int2* tiles; // [ntiles] (tm, tn) in the order the tiles are handed out
   int* status;
 };
 
@@ -120,13 +121,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 
-// Linear index of a lower-triangle tile -> (tm, tn).  Row pair (2a, 2a+1) holds a+1 tiles each.
-__device__ __forceinline__ void tile_coords(int t, int& tm, int& tn) {
-  int a = 0;
-  while ((a + 1) * (a + 2) <= t) ++a;
-  const int rem = t - a * (a + 1);
-  if (rem < a + 1) { tm = 2 * a; tn = rem; }
-  else { tm = 2 * a + 1; tn = rem - (a + 1); }
+// Order in which the lower-triangle tiles (tn <= tm / 2) are handed out: bands of BAND tile
+// rows, and inside a band column by column.  Consecutive tiles -- the ones the persistent CTAs
+// work on at the same time -- then form a compact block of about BAND x (SMs / BAND) tiles that
+// shares its operand panels in L2, instead of a strip that spans every column of X.
+constexpr int BAND = 16;
+__global__ void hessian_tile_order_kernel(int tiles_m, int2* __restrict__ tiles) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  int t = 0;
+  for (int r0 = 0; r0 < tiles_m; r0 += BAND) {
+    const int r1 = min(tiles_m, r0 + BAND);
+    for (int tn = 0; tn <= (r1 - 1) / 2; ++tn)
+      for (int tm = max(r0, 2 * tn); tm < r1; ++tm) tiles[t++] = make_int2(tm, tn);
+  }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -174,8 +181,8 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, Params p) {
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         const int s = u / p.ntiles, t = u - s * p.ntiles;
-        int tm, tn;
-        tile_coords(t, tm, tn);
+        const int2 tc = p.tiles[t];
+        const int tm = tc.x, tn = tc.y;
         const int kb0 = (int)((long long)s * p.kblocks / p.splits), kb1 = (int)((long long)(s + 1) * p.kblocks / p.splits);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -281,8 +288,7 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, Params p) {
 // accumulating, and write the lower-triangle entry together with its mirror image.
 __global__ void __launch_bounds__(256) hessian_reduce_kernel(Params p, int accumulate, float* __restrict__ H) {
   const int t = blockIdx.x;
-  int tm, tn;
-  tile_coords(t, tm, tn);
+  const int tm = p.tiles[t].x, tn = p.tiles[t].y;
   const long long d = p.d_in;
   for (int idx = threadIdx.x; idx < TILE_ELEMS; idx += blockDim.x) {
     const long long r = (long long)tm * BM + idx / BN, c = (long long)tn * BN + idx % BN;
@@ -324,7 +330,7 @@ bool hessian_tc_supported(long long n, long long d_in, long long ldx, const void
 size_t hessian_tc_workspace(long long n, long long d_in) {
   if (d_in < 256 || n < 256) return 0;
   const tc::Plan pl = tc::make_plan(n, d_in);
-  return align_up((size_t)pl.splits * pl.ntiles * tc::TILE_ELEMS * sizeof(float));
+  return align_up((size_t)pl.splits * pl.ntiles * tc::TILE_ELEMS * sizeof(float)) + align_up((size_t)pl.ntiles * sizeof(int2));
 }
 
 cudaError_t launch_hessian_tc(const void* X, long long n, long long d_in, long long ldx, int accumulate, float* H,
@@ -358,6 +364,9 @@ cudaError_t launch_hessian_tc(const void* X, long long n, long long d_in, long l
   Params p{};
   p.n = n; p.d_in = d_in; p.tiles_m = pl.tiles_m; p.ntiles = pl.ntiles; p.splits = pl.splits; p.kblocks = pl.kblocks;
   p.partials = (float*)ws;
+  int2* tiles = (int2*)((char*)ws + align_up((size_t)pl.splits * pl.ntiles * TILE_ELEMS * sizeof(float)));
+  p.tiles = tiles;
+  hessian_tile_order_kernel<<<1, 32, 0, st>>>(pl.tiles_m, tiles);
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
   int dev = 0, sms = 0;
