@@ -60,8 +60,10 @@ Layer make_layer(const float* H, const void* W, cdq_dtype wt, long long d_in, lo
 
 // Workspace of cdq_cd_solve / cdq_layer_loss.
 struct SolveWs {
-  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, total;
+  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, hbuf, ebuf, total;
   long long ldg, d_pad;
+  bool tc;        // H E on the int8 tensor cores
+  int nh, ne, smax;
 };
 SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd) {
   SolveWs w{};
@@ -69,9 +71,15 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   w.ldg = (d_in + 3) / 4 * 4;
   w.d_pad = cd_fast_pad(d_in);
+  w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+  w.nh = with_cd ? kTcGradNH : kTcLossNH; w.ne = with_cd ? kTcGradNE : kTcLossNE; w.smax = with_cd ? kTcGradSmax : kTcLossSmax;
   w.E = take(sizeof(double) * d_in * d_out);
+  if (with_cd || w.tc) w.G = take(sizeof(double) * d_out * w.ldg);
+  if (w.tc) {
+    w.hbuf = take(gemm_tc_h_bytes(d_in, w.nh));
+    w.ebuf = take(gemm_tc_e_bytes(d_in, d_out, w.ne));
+  }
   if (with_cd) {
-    w.G = take(sizeof(double) * d_out * w.ldg);
     w.Qt = take((size_t)d_out * w.ldg);  // transposed codes, same leading dimension as G
     w.hdiag = take(sizeof(float) * w.d_pad);
     w.half_inv = take(sizeof(float) * w.d_pad);
@@ -97,6 +105,13 @@ void note_cuda_error(cudaError_t e, const char* what, int line) {
 
 // CDQ_DEBUG_SYNC=1 in the environment synchronises the device after every step, so that an
 // asynchronous kernel failure is attributed to the step that caused it.
+}  // namespace
+bool gemm_tc_enabled() {
+  static const bool on = [] { const char* e = getenv("CDQ_GEMM"); return !(e && e[0] == 's'); }();
+  return on;
+}
+namespace {
+
 bool debug_sync() {
   static int v = -1;
   if (v < 0) {
@@ -250,8 +265,14 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
 
   // G0 = 2 H (W_hat - W) and the loss at entry
   CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
-  if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, G, L.ldg, col_loss, part, st));
-  else CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, G, L.ldg, col_loss, st));
+  if (L.tc) {
+    CDQ_CUDA(gemm_tc_prepare_h(H, d_in, L.nh, base + L.hbuf, st));
+    CDQ_CUDA(gemm_tc_run(base + L.hbuf, L.nh, E, d_in, d_out, L.ne, L.smax, 2.0, G, L.ldg, col_loss, base + L.ebuf, st));
+  } else if (mode == CDQ_MODE_FAST) {
+    CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, G, L.ldg, col_loss, part, st));
+  } else {
+    CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, G, L.ldg, col_loss, st));
+  }
   CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
   CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, d_out, Qt, L.ldg, st));
   CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
@@ -313,8 +334,15 @@ cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long
   double* col_loss = per_col ? per_col : (double*)(base + L.col_loss);
   double* loss_sum = (double*)(base + L.scalars);
   CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
-  if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, nullptr, 0, col_loss, part, st));
-  else CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, nullptr, 0, col_loss, st));
+  if (L.tc) {
+    CDQ_CUDA(gemm_tc_prepare_h(H, d_in, L.nh, base + L.hbuf, st));
+    CDQ_CUDA(gemm_tc_run(base + L.hbuf, L.nh, E, d_in, d_out, L.ne, L.smax, 1.0, (double*)(base + L.G), L.ldg, col_loss,
+                         base + L.ebuf, st));
+  } else if (mode == CDQ_MODE_FAST) {
+    CDQ_CUDA(launch_gemm_he(H, d_in, d_out, E, nullptr, 0, col_loss, part, st));
+  } else {
+    CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, nullptr, 0, col_loss, st));
+  }
   if (loss) {
     CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
     CDQ_CUDA(cudaMemcpyAsync(loss, loss_sum, sizeof(double), cudaMemcpyDeviceToHost, st));

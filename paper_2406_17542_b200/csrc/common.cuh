@@ -81,6 +81,20 @@ cudaError_t launch_gemm_he(const float* H, long long d_in, long long d_out, cons
 cudaError_t launch_gemm_he_verify(const float* H, long long d_in, long long d_out, const double* E, double* C,
                                   double* G, long long ldg, double* col_loss, cudaStream_t st);
 
+// gemm_i8.cu : C[j, p] = scale * sum_k E[k, j] H[p, k] on the int8 tensor cores from 7-bit slices of
+// both operands (nh slices of H, ne of E, slice pairs up to i + j = smax); C is [d_out, ldc].
+// col_loss (may be NULL): [d_out], e_j^T H e_j.
+bool gemm_tc_supported(long long d_in, long long d_out);
+size_t gemm_tc_h_bytes(long long d_in, int nh);
+size_t gemm_tc_e_bytes(long long d_in, long long d_out, int ne);
+cudaError_t gemm_tc_prepare_h(const float* H, long long d_in, int nh, void* hbuf, cudaStream_t st);
+cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_in, long long d_out, int ne, int smax,
+                        double scale, double* C, long long ldc, double* col_loss, void* ebuf, cudaStream_t st);
+// Slice counts: the gradient needs ~1e-9 of a_j H_pp (see gemm_i8.cu); a loss needs ~1e-7 relative.
+constexpr int kTcGradNH = 6, kTcGradNE = 5, kTcGradSmax = 9;
+constexpr int kTcLossNH = 4, kTcLossNE = 4, kTcLossSmax = 6;
+bool gemm_tc_enabled();   // false when CDQ_GEMM=simt is set in the environment
+
 // cd_kernel.cu
 struct CdCounters {            // lives in the workspace, zeroed by the launcher
   unsigned long long committed;
