@@ -141,7 +141,9 @@ __global__ void fill_gamma_kernel(float* gamma_out, long long d_out) {
 //   OWC only : gammas [n_clip] f64, gam_col [d_out] f64, table [n_clip, d_out] f64,
 //              E [d_in, d_out] f64, loss partials (FAST) or the product H E (VERIFY)
 struct InitWs {
-  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, total;
+  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, total;
+  bool tc;          // losses on the int8 tensor cores
+  long long ldc;
 };
 static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n_clip, cdq_mode mode) {
   InitWs w{};
@@ -159,6 +161,13 @@ static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n
     w.table = take(sizeof(double) * n_clip * d_out);
     w.E = take(sizeof(double) * d_in * d_out);
     w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
+    w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+    w.ldc = (d_in + 3) / 4 * 4;
+    if (w.tc) {
+      w.C = take(sizeof(double) * d_out * w.ldc);
+      w.hbuf = take(gemm_tc_h_bytes(d_in, kTcLossNH));
+      w.ebuf = take(gemm_tc_e_bytes(d_in, d_out, kTcLossNE));
+    }
   }
   w.total = off;
   return w;
@@ -198,6 +207,10 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
     cudaError_t e = cudaMemcpyAsync(gammas, hg, sizeof(double) * n_clip, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return e;
     // the host array must outlive the copy: pageable memcpy is staged before return
+    if (L.tc) {   // the slices of H serve every clipping strength
+      e = gemm_tc_prepare_h(ly.H, d_in, kTcLossNH, base + L.hbuf, st);
+      if (e != cudaSuccess) return e;
+    }
     for (int k = 0; k < n_clip; ++k) {
       ResidualSrc src{};
       src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
@@ -205,7 +218,10 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
       src.g = g; src.d_out = d_out;
       e = launch_residual_f64(src, d_in, E, st);
       if (e != cudaSuccess) return e;
-      if (mode == CDQ_MODE_FAST)
+      if (L.tc)
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, d_out, kTcLossNE, kTcLossSmax, 1.0, (double*)(base + L.C), L.ldc,
+                        table + (long long)k * d_out, base + L.ebuf, st);
+      else if (mode == CDQ_MODE_FAST)
         e = launch_gemm_he(ly.H, d_in, d_out, E, nullptr, 0, table + (long long)k * d_out, part, st);
       else
         e = launch_gemm_he_verify(ly.H, d_in, d_out, E, part, nullptr, 0, table + (long long)k * d_out, st);

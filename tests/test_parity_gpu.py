@@ -83,9 +83,10 @@ def test_small_and_ragged_shapes(d_in, d_out, n, bits, g, mode):
         assert abs(gpu["loss"] - ora["loss"]) <= LOSS_RTOL * max(ora["loss"], 1e-30)
 
 
+@pytest.mark.parametrize("d_in,d_out", [(256, 96), (512, 160)])   # fp64 SIMT losses; int8 tensor-core losses
 @pytest.mark.parametrize("mode", ["verify", "fast"])
-def test_owc_clip_search(mode):
-    cfg = inputs.CONFIGS["C2"].scaled(d_in=256, d_out=96, n=1024, seed=7)
+def test_owc_clip_search(mode, d_in, d_out):
+    cfg = inputs.CONFIGS["C2"].scaled(d_in=d_in, d_out=d_out, n=4 * d_in, seed=7)
     X, W = inputs.make_layer(cfg)
     ora = oracle_pipeline(cfg, X, W)
     gpu = gpu_pipeline(cfg, X, W, mode=mode, H=ora["H"])
