@@ -273,7 +273,8 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   } else {
     CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, G, L.ldg, col_loss, st));
   }
-  CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
+  if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_sum_f64_tree(col_loss, d_out, loss_sum, st));
+  else CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
   CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, d_out, Qt, L.ldg, st));
   CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -344,7 +345,8 @@ cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long
     CDQ_CUDA(launch_gemm_he_verify(H, d_in, d_out, E, part, nullptr, 0, col_loss, st));
   }
   if (loss) {
-    CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
+    if (mode == CDQ_MODE_FAST) CDQ_CUDA(launch_sum_f64_tree(col_loss, d_out, loss_sum, st));
+    else CDQ_CUDA(launch_sum_f64(col_loss, d_out, loss_sum, st));
     CDQ_CUDA(cudaMemcpyAsync(loss, loss_sum, sizeof(double), cudaMemcpyDeviceToHost, st));
     CDQ_CUDA(cudaStreamSynchronize(st));
   }

@@ -7,7 +7,8 @@
 //   r = clamp(rint(q - g / (2 a H_ii)), 0, L).
 // (Variants that were measured and dropped: a chunk-level running minimum with the winner
 // worked out afterwards, a packed fp64 min carrying score and identity, and an integer-pipe
-// fp64 -> fp32 truncation; each made the step slower or no faster on B200.)
+// fp64 -> fp32 truncation, and the packed f32x2 arithmetic of sm_100 for the fp32 part; each made
+// the step slower or no faster on B200.)
 #pragma once
 
 #include "cd_params.cuh"

@@ -115,5 +115,6 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
 cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                              long long steps_per_col, CdCounters* ctr, cudaStream_t st);
 cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st);  // ascending order
+cudaError_t launch_sum_f64_tree(const double* v, long long n, double* out, cudaStream_t st);  // fixed tree order
 
 }  // namespace cdq

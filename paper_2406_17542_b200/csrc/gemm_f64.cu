@@ -200,4 +200,25 @@ cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream
   return cudaGetLastError();
 }
 
+// The same sum by one block in a fixed tree order (reproducible from run to run, not the
+// ascending order): for the production mode, where d_out can be tens of thousands.
+__global__ void __launch_bounds__(1024) sum_f64_tree_kernel(const double* __restrict__ v, long long n,
+                                                            double* __restrict__ out) {
+  __shared__ double red[1024];
+  double s = 0.0;
+  for (long long i = threadIdx.x; i < n; i += 1024) s += v[i];
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = 512; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = red[0];
+}
+
+cudaError_t launch_sum_f64_tree(const double* v, long long n, double* out, cudaStream_t st) {
+  sum_f64_tree_kernel<<<1, 1024, 0, st>>>(v, n, out);
+  return cudaGetLastError();
+}
+
 }  // namespace cdq
