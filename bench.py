@@ -33,7 +33,12 @@ UNIT = "updates/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the descent kernel, from the ncu
 # capture summarised under profiles/ (workload -> bytes); None until a capture exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # cd_fast_kernel, 4096-column capture (1.784 GB) x 16 254 834 / 4 053 277 committed moves
+    "C1": 7.15e9,
+    # cd_tma_kernel, 592-column capture (242.5 GB) x 18 354 343 / 5 450 779 committed moves
+    "C3": 8.17e11,
+}
 
 
 def load_peaks():
