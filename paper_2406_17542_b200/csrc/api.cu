@@ -72,7 +72,10 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   w.ldg = (d_in + 3) / 4 * 4;
   w.d_pad = cd_fast_pad(d_in);
   w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
-  w.nh = with_cd ? kTcGradNH : kTcLossNH; w.ne = with_cd ? kTcGradNE : kTcLossNE; w.smax = with_cd ? kTcGradSmax : kTcLossSmax;
+  // the loss of a descended solution is a sum with heavy cancellation (the descent tunes e against the
+  // large entries of H): it takes the same slice depth as the gradient; the shallower setting serves
+  // the OWC search, whose residuals are plain rounding errors
+  w.nh = kTcGradNH; w.ne = kTcGradNE; w.smax = kTcGradSmax;
   w.E = take(sizeof(double) * d_in * d_out);
   if (with_cd || w.tc) w.G = take(sizeof(double) * d_out * w.ldg);
   if (w.tc) {

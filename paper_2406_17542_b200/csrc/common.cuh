@@ -90,7 +90,8 @@ size_t gemm_tc_e_bytes(long long d_in, long long d_out, int ne);
 cudaError_t gemm_tc_prepare_h(const float* H, long long d_in, int nh, void* hbuf, cudaStream_t st);
 cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_in, long long d_out, int ne, int smax,
                         double scale, double* C, long long ldc, double* col_loss, void* ebuf, cudaStream_t st);
-// Slice counts: the gradient needs ~1e-9 of a_j H_pp (see gemm_i8.cu); a loss needs ~1e-7 relative.
+// Slice counts: the gradient and the loss of a descended solution need ~1e-9 of a_j H_pp (see
+// gemm_i8.cu); the losses of the OWC search (round-to-nearest residuals) need ~1e-7 relative.
 constexpr int kTcGradNH = 6, kTcGradNE = 5, kTcGradSmax = 9;
 constexpr int kTcLossNH = 4, kTcLossNE = 4, kTcLossSmax = 6;
 bool gemm_tc_enabled();   // false when CDQ_GEMM=simt is set in the environment
