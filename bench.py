@@ -104,11 +104,17 @@ class ClockSampler:
 
 
 def kernel_launches(cfg) -> int:
-    """Kernels of the library launched by one step (counted from the launch sequences)."""
-    hessian = 1
-    init = 4 + (1 + 3 * cfg.n_clip if cfg.n_clip > 1 else 0)
-    cd = 8          # residual, gemm, partial sums, total, transpose, diag, descent, transpose
-    loss = 4        # residual, gemm, partial sums, total
+    """Kernels of the library launched by one step (counted from the launch sequences in csrc/)."""
+    tc_h = cfg.x_dtype == "bf16" and cfg.n >= 256 and cfg.d_in >= 256          # tcgen05 Hessian: order, MMA, reduce
+    tc_g = cfg.d_in >= 256 and cfg.d_out >= 128                                  # int8 tensor-core H E
+    hessian = 3 if tc_h else 1
+    prep_h = 2                                                                   # row exponents, slices of H
+    he = 5 if tc_g else 2                # column max, exponents, slices of E^T, GEMM, column dot | GEMM, partial sums
+    init = 5                                                                     # min/max x2, gamma fill or argmin, scale/zero, codes
+    if cfg.n_clip > 1:
+        init += (prep_h if tc_g else 0) + cfg.n_clip * (1 + he)                  # per gamma: residual + H E
+    cd = 1 + (prep_h if tc_g else 0) + he + 1 + 1 + 1 + 1 + 1                    # residual, H E, sum, transpose, diag, descent, transpose
+    loss = 1 + (prep_h if tc_g else 0) + he + 1                                  # residual, H E, sum
     return hessian + init + cd + loss
 
 
