@@ -29,12 +29,15 @@
  *     Arguments are validated before any launch.  A device-side wait that
  *     exceeds its bound is reported as CDQ_ERR_TIMEOUT by the next call that
  *     synchronises (cdq_last_device_status reads it explicitly).
- *   - Two arithmetic modes.  CDQ_MODE_FAST is the production path: fp32 H,
- *     fp32 candidate scoring, gradient kept in fp64, tensor cores for the
- *     Hessian.  CDQ_MODE_FP64_VERIFY runs plain fp64 kernels that follow a
- *     fixed summation order (ascending index, no fused multiply-add) so that
- *     codes can be compared bit for bit with a CPU implementation of the same
- *     steps; it is meant for small layers.
+ *   - Two arithmetic modes.  CDQ_MODE_FAST is the production path: fp32 H, tensor cores for
+ *     the Hessian (bf16) and for the products H (W_hat - W) (exact int8 slices, summed in fp64),
+ *     the gradient of the descent kept in fp64 and the candidate scores in fp32.  Grouped grids
+ *     whose group size is not a multiple of 4, and layers longer than 18432 inputs, run their
+ *     descent with the fp64 kernel of the other mode.  CDQ_MODE_FP64_VERIFY runs plain fp64
+ *     kernels that follow a fixed summation order (ascending index, no fused multiply-add) so
+ *     that codes can be compared bit for bit with a CPU implementation of the same steps; it is
+ *     meant for small layers.
+ *   - H must be finite; the descent multiplies rows of H by a zero step in its first sweep.
  */
 #ifndef CDQ_H_
 #define CDQ_H_
