@@ -58,6 +58,8 @@ def _load():
     lib.cdqo_gamma.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double]
     lib.cdqo_hessian.argtypes = [_dp, _i64, _i64, ctypes.c_double, _dp, _fp]
     lib.cdqo_hessian_entries.argtypes = [_dp, _i64, _i64, _i64p, _i64p, _i64, _dp]
+    lib.cdqo_owc_cd.argtypes = [_dp, _i64, _i64, _fp, ctypes.c_int, _i64, ctypes.c_int, ctypes.c_double,
+                                ctypes.c_double, _i64, _fp, _fp, _u8p, _ip, _i64p, _dp, _dp]
     lib.cdqo_init_rtn.argtypes = [_dp, _i64, _i64, _fp, ctypes.c_int, _i64, ctypes.c_int,
                                   ctypes.c_double, ctypes.c_double, _fp, _fp, _u8p, _ip, _dp]
     lib.cdqo_gradient.argtypes = [_fp, _dp, _i64, _i64, _i64, _fp, _fp, _u8p, _dp]
@@ -152,6 +154,28 @@ def init_rtn(W, bits: int, group_size: int = 0, n_clip: int = 1, clip_lo: float 
     assert rc == 0, rc
     return {"scale": scale, "zero": zero, "Q": Q, "gamma_idx": gidx,
             "gamma": gamma_grid(n_clip, clip_lo, clip_hi)[gidx], "loss_table": table}
+
+
+def owc_cd(H, W, bits: int, group_size: int, n_clip: int, clip_lo: float, clip_hi: float, steps: int) -> dict:
+    """OWC-CD (Algorithm 3): greedy descent over the clipping strengths of a column's groups,
+    every group starting at the last grid point; `steps` changes per column at most."""
+    Hf, W = _f32(H), _f64(W)
+    d_in, d_out = W.shape
+    g = group_size if group_size > 0 else d_in
+    ng = d_in // g
+    scale = np.empty((ng, d_out), dtype=np.float32)
+    zero = np.empty((ng, d_out), dtype=np.float32)
+    Q = np.empty((d_in, d_out), dtype=np.uint8)
+    gidx = np.zeros((ng, d_out), dtype=np.int32)
+    moves = np.zeros(d_out, dtype=np.int64)
+    lb = np.zeros(d_out, dtype=np.float64)
+    la = np.zeros(d_out, dtype=np.float64)
+    rc = _load().cdqo_owc_cd(_ptr(W, _dp), d_in, d_out, _ptr(Hf, _fp), int(bits), int(group_size), int(n_clip),
+                             float(clip_lo), float(clip_hi), int(steps), _ptr(scale, _fp), _ptr(zero, _fp),
+                             _ptr(Q, _u8p), _ptr(gidx, _ip), _ptr(moves, _i64p), _ptr(lb, _dp), _ptr(la, _dp))
+    assert rc == 0, rc
+    return {"scale": scale, "zero": zero, "Q": Q, "gamma_idx": gidx, "moves": moves,
+            "loss_before": lb, "loss_after": la}
 
 
 def gradient(H, W, scale, zero, Q, group_size: int = 0) -> np.ndarray:

@@ -15,6 +15,8 @@
  *   - greedy coordinate descent                    (Algorithm 1 lines 4-8;
  *     Algorithm 4 for sub-channel grids)
  *   - the layer loss  sum_j e_j^T H e_j            (Eq. 1 written with H)
+ *   - OWC-CD: greedy descent over per-group clipping strengths (Algorithm 3;
+ *     its readings are listed above cdqo_owc_cd)
  *
  * Formulation.  Algorithm 1 works in code units (g = 2H(q - (w-b)/a), the
  * printed decrease (r-q_i)^2 H_ii + (r-q_i) g_i is the loss change divided by
@@ -47,7 +49,10 @@
  * Delta against the loss recomputed from X; incremental G against a fresh
  * 2H(w_hat-w); monotone loss; closed-form coordinate optimum against the level
  * scan; diagonal H => no move; gamma = 1 => MinMax; code-unit Algorithm 4 ==
- * weight-unit picks; local optimality at convergence; d_in = 1.
+ * weight-unit picks; local optimality at convergence; d_in = 1.  OWC-CD:
+ * tracked loss against the loss recomputed from X; one group == the OWC grid
+ * search; brute force over all assignments of grid points to groups; first
+ * change == best single-group change; convergence == no improving change.
  * Parity unpinned: anything that depends on the paper's (unstated) lambda.
  */
 #include <math.h>
@@ -439,5 +444,131 @@ int cdqo_layer_loss(const float* H, const double* W, i64 d_in, i64 d_out,
   if (per_col) memcpy(per_col, col_loss, sizeof(double) * d_out);
   *total = sum;
   free(col_loss);
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* OWC-CD: greedy coordinate descent over the clipping strengths of the      */
+/* groups of a column (Algorithm 3, "Coordinate Descent for Optimal Weight   */
+/* Clipping", sub-channel section).                                          */
+/*                                                                           */
+/* State per column: one grid index per group, and G = 2 H e with            */
+/* e = w_hat - w (the vector the algorithm calls v; see the sign note).      */
+/* Table: for every group t and grid point k the residual of that group      */
+/* under Eq. 2 with gamma_k (Algorithm 3 lines 2-6).                         */
+/* Step: for every group t and every k other than its current index, with    */
+/* delta = residual(t, k) - residual(t, current) (a vector over the group),  */
+/*     change(t, k) = delta^T H_tt delta + delta^T G_t        (line 11)      */
+/* take the most negative one, then G <- G + 2 H[:, t] delta  (line 12)      */
+/* and set the group's index to k (line 13).                                 */
+/*                                                                           */
+/* Readings:                                                                 */
+/*  - sign: the paper defines the table entry as w - w_hat and v as          */
+/*    -2 H (w_hat - w) but adds v^T (Delta_old - Delta_new); with those      */
+/*    signs the linear term would be minus the true one.  The change of the  */
+/*    quadratic loss for e -> e + delta is delta^T H delta + 2 e^T H delta,  */
+/*    which is what is computed here, and the update of line 12 is           */
+/*    consistent with it;                                                    */
+/*  - start (line 7 says only "initialize"): every group starts at the last  */
+/*    grid point (the largest gamma; MinMax when clip_hi = 1);               */
+/*  - ties: lowest group, then lowest grid index; a change is made only if   */
+/*    it strictly lowers the loss, otherwise the column is finished;         */
+/*  - T: `steps` per column (the paper's experiments use d_in / g).          */
+/* Sums run in ascending index order, no fused multiply-add.                 */
+/*                                                                           */
+/* W: [d_in, d_out] fp64 (widened), H fp32.  Outputs: scale, zero            */
+/* [d_in/g, d_out] fp32, Q [d_in, d_out] u8, gamma_idx [d_in/g, d_out],      */
+/* moves / loss_before / loss_after [d_out] (each may be NULL).              */
+/* ------------------------------------------------------------------------ */
+int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
+                i64 group_size, int n_clip, double clip_lo, double clip_hi,
+                i64 steps, float* scale, float* zero, uint8_t* Q, int* gamma_idx,
+                i64* moves, double* loss_before, double* loss_after) {
+  if (!W || !H || !scale || !zero || !Q || bits < 1 || bits > 8 || d_in <= 0 || d_out <= 0 || n_clip < 1)
+    return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g) return 2;
+  const i64 ng = d_in / g;
+  const int L = (1 << bits) - 1;
+  const int nk = n_clip;
+#pragma omp parallel
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* tab = (double*)malloc(sizeof(double) * (size_t)nk * d_in); /* [k][i]: residual of coordinate i under gamma_k */
+    double* G = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    double* he = (double*)malloc(sizeof(double) * d_in);
+    double* delta = (double*)malloc(sizeof(double) * g);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+    int* cur = (int*)malloc(sizeof(int) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) w[i] = W[i * d_out + j];
+      /* residual table (lines 2-6) */
+      for (int k = 0; k < nk; ++k) {
+        const double gamma = cdqo_gamma(k, nk, clip_lo, clip_hi);
+        for (i64 t = 0; t < ng; ++t)
+          grid_rtn_group(w + t * g, g, L, gamma, a + t, b + t, q + t * g);
+        residual(w, q, a, b, d_in, g, tab + (size_t)k * d_in);
+      }
+      /* start (line 7) and G = 2 H e (lines 8-9) */
+      for (i64 t = 0; t < ng; ++t) cur[t] = nk - 1;
+      for (i64 i = 0; i < d_in; ++i) e[i] = tab[(size_t)(nk - 1) * d_in + i];
+      double loss = quad_form(H, e, d_in, he);
+      for (i64 i = 0; i < d_in; ++i) G[i] = 2.0 * he[i];
+      if (loss_before) loss_before[j] = loss;
+      i64 nmoves = 0;
+      for (i64 step = 0; step < steps; ++step) {
+        double best = 0.0;
+        i64 bt = -1;
+        int bk = 0;
+        for (i64 t = 0; t < ng; ++t) {
+          const double* old = tab + (size_t)cur[t] * d_in + t * g;
+          for (int k = 0; k < nk; ++k) {
+            if (k == cur[t]) continue;
+            const double* cand = tab + (size_t)k * d_in + t * g;
+            for (i64 p = 0; p < g; ++p) delta[p] = cand[p] - old[p];
+            double quad = 0.0, lin = 0.0;
+            for (i64 p = 0; p < g; ++p) {
+              const float* row = H + (t * g + p) * d_in + t * g;
+              double acc = 0.0;
+              for (i64 r = 0; r < g; ++r) acc = acc + (double)row[r] * delta[r];
+              quad = quad + delta[p] * acc;
+              lin = lin + delta[p] * G[t * g + p];
+            }
+            const double change = quad + lin;
+            if (change < best) { best = change; bt = t; bk = k; }
+          }
+        }
+        if (bt < 0) break;
+        const double* old = tab + (size_t)cur[bt] * d_in + bt * g;
+        const double* cand = tab + (size_t)bk * d_in + bt * g;
+        for (i64 p = 0; p < g; ++p) delta[p] = cand[p] - old[p];
+        for (i64 i = 0; i < d_in; ++i) {
+          const float* row = H + i * d_in + bt * g;
+          double acc = 0.0;
+          for (i64 r = 0; r < g; ++r) acc = acc + (double)row[r] * delta[r];
+          G[i] = G[i] + 2.0 * acc;
+        }
+        cur[bt] = bk;
+        loss = loss + best;
+        ++nmoves;
+      }
+      /* emit the grid and the codes of the chosen strengths */
+      for (i64 t = 0; t < ng; ++t) {
+        const double gamma = cdqo_gamma(cur[t], nk, clip_lo, clip_hi);
+        grid_rtn_group(w + t * g, g, L, gamma, a + t, b + t, q + t * g);
+        scale[t * d_out + j] = a[t];
+        zero[t * d_out + j] = b[t];
+        if (gamma_idx) gamma_idx[t * d_out + j] = cur[t];
+      }
+      for (i64 i = 0; i < d_in; ++i) Q[i * d_out + j] = q[i];
+      if (moves) moves[j] = nmoves;
+      if (loss_after) loss_after[j] = loss;
+    }
+    free(w); free(tab); free(G); free(e); free(he); free(delta); free(q); free(a); free(b); free(cur);
+  }
   return 0;
 }

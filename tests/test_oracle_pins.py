@@ -334,3 +334,97 @@ def test_tie_break_lowest_coordinate_then_lowest_level():
     W2 = np.array([[1.5], [0.0]], dtype=np.float32)        # levels 1 and 2 tie for coordinate 0
     res = oracle.cd_solve(H, W2, 2, a, b, Q0, steps_per_col=1, trace_col=0)
     assert (res["trace"]["i"][0], res["trace"]["r"][0]) == (0, 1)
+
+
+# ---------------------------------------------------------------- OWC-CD (Algorithm 3)
+def _group_grids(W, H32, bits, g, grid):
+    """Per group t and grid point k: (a, b, q) of Eq. 2 for every column, from the pinned per-channel
+    routine on the group's rows (a two-point grid with both points at gamma_k forces that gamma)."""
+    d_in, d_out = W.shape
+    out = {}
+    for t in range(d_in // g):
+        rows = slice(t * g, (t + 1) * g)
+        Hs = np.ascontiguousarray(H32[rows, rows])
+        for k, gam in enumerate(grid):
+            r = oracle.init_rtn(W[rows], bits, 0, n_clip=2, clip_lo=float(gam), clip_hi=float(gam), H=Hs)
+            out[(t, k)] = (r["scale"][0], r["zero"][0], r["Q"])
+    return out
+
+
+def _assemble(grids, choice, d_in, d_out, g):
+    """Layer grid and codes when group t of column j uses grid point choice[t, j]."""
+    ng = d_in // g
+    scale = np.empty((ng, d_out), np.float32); zero = np.empty((ng, d_out), np.float32)
+    Q = np.empty((d_in, d_out), np.uint8)
+    for t in range(ng):
+        for j in range(d_out):
+            a, b, q = grids[(t, int(choice[t, j]))]
+            scale[t, j] = a[j]; zero[t, j] = b[j]; Q[t * g:(t + 1) * g, j] = q[:, j]
+    return scale, zero, Q
+
+
+def test_owc_cd_tracked_loss_is_the_loss_from_x_and_never_rises():
+    d_in, d_out, g, bits = 32, 6, 8, 3
+    X, W = _layer(41, 200, d_in, d_out, feat_sigma=1.2)
+    _, H32 = oracle.hessian(X)
+    for steps in (0, 1, 2, d_in // g, 50):
+        r = oracle.owc_cd(H32, W, bits, g, 6, 0.5, 1.0, steps)
+        direct = _direct_loss(X, W, r["scale"], r["zero"], r["Q"])
+        # the running loss (start + predicted changes) is the loss recomputed from X: pins the
+        # sign and the factor 2 of the linear term and the block of H in the quadratic term
+        np.testing.assert_allclose(r["loss_after"], direct, rtol=1e-5)      # H is fp32: X^T X rounded
+        _, per = oracle.layer_loss(H32, W, r["scale"], r["zero"], r["Q"], g)
+        np.testing.assert_allclose(r["loss_after"], per, rtol=1e-10)
+        assert (r["loss_after"] <= r["loss_before"]).all() and (r["moves"] <= steps).all()
+    # step 0 is MinMax when the grid ends at 1
+    r0 = oracle.owc_cd(H32, W, bits, g, 6, 0.5, 1.0, 0)
+    mm = oracle.init_rtn(W, bits, g)
+    assert np.array_equal(r0["Q"], mm["Q"]) and np.array_equal(r0["scale"], mm["scale"])
+
+
+def test_owc_cd_with_one_group_is_the_owc_grid_search():
+    d_in, d_out, bits = 16, 12, 3
+    X, W = _layer(42, 120, d_in, d_out)
+    _, H32 = oracle.hessian(X)
+    owc = oracle.init_rtn(W, bits, 0, n_clip=8, clip_lo=0.4, clip_hi=1.0, H=H32, want_loss_table=True)
+    r = oracle.owc_cd(H32, W, bits, 0, 8, 0.4, 1.0, 1)
+    # one change from the last grid point lands on the grid search's minimiser
+    assert np.array_equal(r["gamma_idx"][0], owc["gamma_idx"])
+    assert np.array_equal(r["Q"], owc["Q"]) and np.array_equal(r["scale"], owc["scale"])
+    np.testing.assert_allclose(r["loss_after"], owc["loss_table"].min(axis=0), rtol=1e-10)
+
+
+def test_owc_cd_against_brute_force_over_all_assignments():
+    d_in, d_out, g, bits, nk = 12, 5, 4, 2, 4
+    X, W = _layer(43, 90, d_in, d_out, feat_sigma=1.0)
+    _, H32 = oracle.hessian(X)
+    grid = oracle.gamma_grid(nk, 0.5, 1.0)
+    grids = _group_grids(W, H32, bits, g, grid)
+    ng = d_in // g
+    losses = {}
+    for combo in itertools.product(range(nk), repeat=ng):
+        choice = np.repeat(np.array(combo)[:, None], d_out, axis=1)
+        s, z, Q = _assemble(grids, choice, d_in, d_out, g)
+        losses[combo] = oracle.layer_loss(H32, W, s, z, Q, g)[1]
+    exact = np.min(np.stack(list(losses.values())), axis=0)
+    start = losses[(nk - 1,) * ng]
+    r = oracle.owc_cd(H32, W, bits, g, nk, 0.5, 1.0, 100)
+    assert (exact <= r["loss_after"] * (1 + 1e-12)).all() and (r["loss_after"] <= start * (1 + 1e-12)).all()
+    for j in range(d_out):
+        combo = tuple(int(v) for v in r["gamma_idx"][:, j])
+        np.testing.assert_allclose(r["loss_after"][j], losses[combo][j], rtol=1e-10)
+        # converged: no single group change lowers the loss
+        for t in range(ng):
+            for k in range(nk):
+                other = combo[:t] + (k,) + combo[t + 1:]
+                assert losses[other][j] >= losses[combo][j] * (1 - 1e-12)
+    # the first change is the best single-group change from the start
+    r1 = oracle.owc_cd(H32, W, bits, g, nk, 0.5, 1.0, 1)
+    for j in range(d_out):
+        singles = {(t, k): losses[tuple(k if u == t else nk - 1 for u in range(ng))][j]
+                   for t in range(ng) for k in range(nk - 1)}
+        (bt, bk), bl = min(singles.items(), key=lambda kv: (kv[1], kv[0]))
+        if bl < start[j]:
+            assert r1["moves"][j] == 1 and int(r1["gamma_idx"][bt, j]) == bk
+        else:
+            assert r1["moves"][j] == 0
