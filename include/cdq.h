@@ -66,7 +66,8 @@ typedef enum {
   CDQ_CALL_HESSIAN = 0,
   CDQ_CALL_INIT_RTN = 1,
   CDQ_CALL_CD_SOLVE = 2,
-  CDQ_CALL_LAYER_LOSS = 3
+  CDQ_CALL_LAYER_LOSS = 3,
+  CDQ_CALL_INIT_OWC_CD = 4
 } cdq_call;
 
 /* Quantization grid (paper: c in "Notation"; group size g in the sub-channel
@@ -126,6 +127,37 @@ cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d
                         const float* H, const cdq_grid_desc* grid, float* scale, float* zero,
                         unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws,
                         size_t ws_bytes, void* stream);
+
+typedef struct {
+  unsigned long long moves; /* changes of a group's clipping strength, over all columns */
+  double loss_before;       /* sum_j e_j^T H e_j with every group at the last grid point  */
+  double loss_after;        /* the same at the chosen strengths (start + changes made)    */
+} cdq_owc_cd_stats;
+
+/*
+ * Grid and round-to-nearest codes with one clipping strength per GROUP, chosen by greedy
+ * coordinate descent over the groups (paper: Algorithm 3, "Coordinate Descent for Optimal
+ * Weight Clipping"; Eq. 2 per group).  Every group of a column starts at the last point of
+ * the grid Gamma (its largest strength; MinMax when clip_hi = 1).  A step evaluates, for every
+ * group t and grid point k, the change of the column loss
+ *     delta^T H_tt delta + delta^T (2 H e)_t,   delta = residual(t, k) - residual(t, current),
+ * makes the change that lowers the loss most (ties: lowest group, then lowest grid index), and
+ * stops when no change lowers it or after `steps` changes (steps <= 0: d_in / g, the paper's
+ * setting).  The sign of the linear term follows the algebra of the quadratic loss; the
+ * algorithm box of the paper prints it with the opposite sign of its own definitions.
+ *   grid       n_clip >= 2; group_size 0 means one group per column, which makes one step the
+ *              plain OWC grid search.
+ *   scale,zero [d_in/g, d_out] fp32 out.    Q [d_in, d_out] u8 out.
+ *   gamma_out  [d_in/g, d_out] fp32 out, chosen strengths; may be NULL.
+ *   stats      host pointer, may be NULL (then the call does not synchronise).
+ * fp64 in both modes; VERIFY sums in ascending order without fused multiply-add
+ * (bit-reproducible against a CPU statement of the steps), FAST tabulates H_tt r per grid point
+ * once per column so that a step costs dot products of length g.
+ */
+cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                           const float* H, const cdq_grid_desc* grid, long long steps, float* scale,
+                           float* zero, unsigned char* Q, float* gamma_out, cdq_owc_cd_stats* stats,
+                           cdq_mode mode, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Greedy coordinate descent on every column (paper: Algorithm 1; Algorithm 4

@@ -21,10 +21,10 @@ STATUS_NAMES = {0: "CDQ_OK", 1: "CDQ_ERR_INVALID_ARG", 2: "CDQ_ERR_SHAPE", 3: "C
                 4: "CDQ_ERR_WORKSPACE", 5: "CDQ_ERR_CUDA", 6: "CDQ_ERR_TIMEOUT"}
 CDQ_F32, CDQ_BF16 = 0, 1
 MODE_FAST, MODE_FP64_VERIFY = 0, 1
-CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS = 0, 1, 2, 3
+CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD = 0, 1, 2, 3, 4
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_cd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
+EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version"]
 
@@ -44,6 +44,10 @@ class cdq_cd_stats(ctypes.Structure):
     _fields_ = [("steps", ctypes.c_ulonglong), ("committed", ctypes.c_ulonglong),
                 ("columns_converged", ctypes.c_ulonglong), ("loss_before", ctypes.c_double),
                 ("loss_after", ctypes.c_double), ("kernel_ms", ctypes.c_double)]
+
+
+class cdq_owc_cd_stats(ctypes.Structure):
+    _fields_ = [("moves", ctypes.c_ulonglong), ("loss_before", ctypes.c_double), ("loss_after", ctypes.c_double)]
 
 
 @dataclass
@@ -80,6 +84,9 @@ def load():
     lib.cdq_hessian.argtypes = [vp, ci, ll, ll, ll, cf, ci, vp, ci, vp, sz, vp]
     lib.cdq_init_rtn.restype = ci
     lib.cdq_init_rtn.argtypes = [vp, ci, ll, ll, ll, vp, gp, vp, vp, vp, vp, ci, vp, sz, vp]
+    lib.cdq_init_owc_cd.restype = ci
+    lib.cdq_init_owc_cd.argtypes = [vp, ci, ll, ll, ll, vp, gp, ll, vp, vp, vp, vp, ctypes.POINTER(cdq_owc_cd_stats),
+                                    ci, vp, sz, vp]
     lib.cdq_cd_solve.restype = ci
     lib.cdq_cd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_layer_loss.restype = ci
@@ -178,6 +185,33 @@ def cdq_init_rtn(W: torch.Tensor, grid: Grid, H: torch.Tensor | None = None, mod
                              zero.data_ptr(), Q.data_ptr(), gamma.data_ptr(), _MODES[mode], wptr, wbytes, _stream())
     _check(st, "cdq_init_rtn")
     return scale, zero, Q, gamma
+
+
+def cdq_init_owc_cd(W: torch.Tensor, grid: Grid, H: torch.Tensor, steps: int = 0, mode="fast",
+                    ws: Workspace | None = None):
+    """OWC-CD (Algorithm 3): one clipping strength per group, chosen by greedy descent over the groups.
+
+    Returns (scale, zero, Q, gamma [d_in/g, d_out] f32, stats dict)."""
+    _need_cuda(W, H)
+    assert W.dim() == 2 and W.stride(1) == 1 and H.is_contiguous() and H.dtype == torch.float32
+    d_in, d_out = W.shape
+    g = grid.group_size if grid.group_size > 0 else d_in
+    ng = max(d_in // g, 1)
+    dev = W.device
+    scale = torch.empty((ng, d_out), dtype=torch.float32, device=dev)
+    zero = torch.empty((ng, d_out), dtype=torch.float32, device=dev)
+    Q = torch.empty((d_in, d_out), dtype=torch.uint8, device=dev)
+    gamma = torch.empty((ng, d_out), dtype=torch.float32, device=dev)
+    gd = grid.c()
+    stats = cdq_owc_cd_stats()
+    ws = ws or _default_ws
+    wptr, wbytes = ws.get(workspace_bytes(CALL_INIT_OWC_CD, 0, d_in, d_out, grid, mode), dev)
+    st = load().cdq_init_owc_cd(W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), H.data_ptr(), ctypes.byref(gd),
+                                int(steps), scale.data_ptr(), zero.data_ptr(), Q.data_ptr(), gamma.data_ptr(),
+                                ctypes.byref(stats), _MODES[mode], wptr, wbytes, _stream())
+    _check(st, "cdq_init_owc_cd")
+    return scale, zero, Q, gamma, {"moves": stats.moves, "loss_before": stats.loss_before,
+                                   "loss_after": stats.loss_after}
 
 
 def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,

@@ -189,6 +189,12 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
       if (g < 1 || d_in % g) return 0;
       return init_rtn_workspace(d_in, d_out, g, grid->n_clip, mode);
     }
+    case CDQ_CALL_INIT_OWC_CD: {
+      if (!grid || d_out < 1 || grid->n_clip < 2 || grid->n_clip > 256) return 0;
+      const long long g = grid->group_size > 0 ? grid->group_size : d_in;
+      if (g < 1 || d_in % g) return 0;
+      return owc_cd_workspace(d_in, d_out, g, grid->n_clip);
+    }
     case CDQ_CALL_CD_SOLVE:
       if (d_out < 1) return 0;
       return solve_ws_layout(d_in, d_out, mode, true).total;
@@ -237,6 +243,29 @@ cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d
   s = check_ws(ws, ws_bytes, init_rtn_workspace(d_in, d_out, ly.g, grid->n_clip, mode));
   if (s != CDQ_OK) return s;
   CDQ_CUDA(launch_init_rtn(ly, *grid, scale, zero, Q, gamma_out, mode, ws, (cudaStream_t)stream));
+  return CDQ_OK;
+}
+
+cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw, const float* H,
+                           const cdq_grid_desc* grid, long long steps, float* scale, float* zero, unsigned char* Q,
+                           float* gamma_out, cdq_owc_cd_stats* stats, cdq_mode mode, void* ws, size_t ws_bytes,
+                           void* stream) {
+  if (!W || !H || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode)) return CDQ_ERR_INVALID_ARG;
+  cdq_status s = check_layer_shape(d_in, d_out, ldw);
+  if (s != CDQ_OK) return s;
+  s = check_grid(grid, d_in);
+  if (s != CDQ_OK) return s;
+  if (grid->n_clip < 2) return CDQ_ERR_INVALID_ARG;
+  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, nullptr, nullptr);
+  if (ly.ng > 65535) return CDQ_ERR_UNSUPPORTED;
+  s = check_ws(ws, ws_bytes, owc_cd_workspace(d_in, d_out, ly.g, grid->n_clip));
+  if (s != CDQ_OK) return s;
+  if (steps <= 0) steps = ly.ng;
+  unsigned long long moves = 0;
+  double lb = 0.0, la = 0.0;
+  CDQ_CUDA(launch_owc_cd(ly, *grid, steps, scale, zero, Q, gamma_out, mode, ws, stats ? &moves : nullptr,
+                         stats ? &lb : nullptr, stats ? &la : nullptr, (cudaStream_t)stream));
+  if (stats) { stats->moves = moves; stats->loss_before = lb; stats->loss_after = la; }
   return CDQ_OK;
 }
 

@@ -59,6 +59,14 @@ size_t init_rtn_workspace(long long d_in, long long d_out, long long g, int n_cl
 cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* scale, float* zero,
                             unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws, cudaStream_t st);
 
+cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* mn, float* mx, cudaStream_t st);
+
+// owc_cd.cu : greedy descent over per-group clipping strengths (paper: Algorithm 3)
+size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip);
+cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long steps, float* scale, float* zero,
+                          unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws, unsigned long long* host_moves,
+                          double* host_before, double* host_after, cudaStream_t st);
+
 // Residual E = W_hat - W in fp64, [d_in, d_out] row-major, either from stored codes or, for
 // the OWC search, from per-group min/max and one clipping strength (codes formed on the fly).
 struct ResidualSrc {

@@ -136,6 +136,16 @@ __global__ void fill_gamma_kernel(float* gamma_out, long long d_out) {
   if (j < d_out) gamma_out[j] = 1.0f;
 }
 
+// Group minima and maxima of every column: mn, mx [ng, d_out]; pmn, pmx [ng * ceil(g / 256), d_out] scratch.
+cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* mn, float* mx, cudaStream_t st) {
+  const long long cpg = (ly.g + kChunkRows - 1) / kChunkRows;
+  const unsigned bx = (unsigned)((ly.d_out + 127) / 128);
+  minmax_partial_kernel<<<dim3(bx, (unsigned)(ly.ng * cpg)), 128, 0, st>>>(ly.W, ly.wt, ly.d_in, ly.d_out, ly.ldw, ly.g,
+                                                                            cpg, pmn, pmx);
+  minmax_final_kernel<<<dim3(bx, (unsigned)ly.ng), 128, 0, st>>>(pmn, pmx, ly.ng, ly.d_out, cpg, mn, mx);
+  return cudaGetLastError();
+}
+
 // Workspace layout (all blocks 256-byte aligned):
 //   pmn, pmx : [ng*cpg, d_out] f32     mn, mx : [ng, d_out] f32
 //   OWC only : gammas [n_clip] f64, gam_col [d_out] f64, table [n_clip, d_out] f64,

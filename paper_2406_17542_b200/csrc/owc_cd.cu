@@ -1,0 +1,371 @@
+// OWC-CD: greedy coordinate descent over the clipping strengths of a column's groups (paper:
+// Algorithm 3, "Coordinate Descent for Optimal Weight Clipping").
+//
+// Per column j: every group t holds a grid index cur[t] (start: the last grid point), the state is
+// G = 2 H e with e = w_hat - w, and one step changes the strength of the one group whose change
+// lowers the loss most:
+//     delta = r(t, k) - r(t, cur[t])           r(t, k): residual of group t under gamma_k (Eq. 2)
+//     change(t, k) = delta^T H_tt delta + delta^T G_t
+//     G <- G + 2 H[:, t] delta
+// (the sign convention is the one under which the change is the true change of the quadratic
+// loss; the paper's box has the linear term with the opposite sign of its own definitions).
+// Ties go to the lowest group, then the lowest grid index; a change must strictly lower the loss.
+//
+// One CTA per column at a time (columns handed out by an atomic counter), fp64 throughout.  The
+// residual table r(., k) of the column is built once in a per-CTA scratch area.
+//   VERIFY: every sum in ascending index order without fused multiply-add, one thread per output,
+//           so that indices and codes can be compared bit for bit with a CPU statement of the steps.
+//   FAST:   M(k) = H_tt r(t, k) is tabulated once per column, after which a step needs only
+//           dot products of length g:  delta^T H_tt delta = r_k.M_k - 2 r_k.M_c + r_c.M_c;
+//           one warp per dot product, lanes across the group.
+#include "common.cuh"
+
+namespace cdq {
+namespace owc {
+
+constexpr int NT = 256;
+
+struct Counters {
+  int next_col;
+  int pad;
+  unsigned long long moves;
+};
+
+struct Params {
+  const float* H;
+  const void* W;
+  cdq_dtype wt;
+  long long d_in, d_out, ldw, g, ng;
+  int L, nk;
+  const double* gammas;   // [nk]
+  const float* mn;        // [ng, d_out] group minima
+  const float* mx;        // [ng, d_out] group maxima
+  long long steps;
+  float* scale;           // [ng, d_out]
+  float* zero;            // [ng, d_out]
+  unsigned char* Q;       // [d_in, d_out]
+  float* gamma_out;       // [ng, d_out] or NULL
+  double* scratch;        // per CTA: R [nk, d_in], M [nk, d_in], G [d_in], S [max(ng * nk, g)]
+  size_t scratch_per_cta; // doubles
+  int* cur;               // per CTA: [ng]
+  double* col_before;     // [d_out]
+  double* col_after;      // [d_out]
+  Counters* ctr;
+};
+
+// Residual a q + b - w of one weight under clipping strength gamma (Eq. 2; the arithmetic of
+// residual_kernel in init_rtn.cu).  Also returns the code and the grid through the pointers.
+__device__ __forceinline__ double resid(double w, double lo, double hi, double gamma, int L, float* a_out,
+                                        unsigned char* q_out) {
+  const float a32 = (float)__ddiv_rn(__dmul_rn(gamma, __dadd_rn(hi, -lo)), (double)L);
+  const double a = (double)a32;
+  double q = 0.0;
+  if (a32 > 0.f) {
+    q = rint(__ddiv_rn(__dadd_rn(w, -lo), a));
+    q = q < 0.0 ? 0.0 : q;
+    q = q > (double)L ? (double)L : q;
+  }
+  if (a_out) *a_out = a32;
+  if (q_out) *q_out = (unsigned char)q;
+  return __dadd_rn(__dadd_rn(__dmul_rn(a, q), lo), -w);
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+template <bool VERIFY>
+__global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
+  __shared__ int s_col;
+  __shared__ double s_val[NT];
+  __shared__ int s_idx[NT];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
+  const long long d_in = p.d_in, g = p.g, ng = p.ng;
+  const int nk = p.nk;
+  double* R = p.scratch + (size_t)blockIdx.x * p.scratch_per_cta;   // [nk, d_in] residuals
+  double* M = R + (size_t)nk * d_in;                                 // [nk, d_in] H_tt r (FAST), H e (VERIFY, row 0)
+  double* G = M + (size_t)nk * d_in;                                 // [d_in]
+  double* S = G + d_in;                                              // [max(ng * nk, g)] scores / delta
+  int* cur = p.cur + (size_t)blockIdx.x * ng;
+  unsigned long long my_moves = 0;
+
+  for (;;) {
+    __syncthreads();
+    if (tid == 0) s_col = atomicAdd(&p.ctr->next_col, 1);
+    __syncthreads();
+    const long long j = s_col;
+    if (j >= p.d_out) break;
+
+    // ---- residual table (Algorithm 3 lines 2-6) and start (line 7) ----
+    for (long long idx = tid; idx < (long long)nk * d_in; idx += NT) {
+      const int k = (int)(idx / d_in);
+      const long long i = idx - (long long)k * d_in, t = i / g;
+      R[idx] = resid(load_w(p.W, p.wt, i * p.ldw + j), (double)p.mn[t * p.d_out + j], (double)p.mx[t * p.d_out + j],
+                     p.gammas[k], p.L, nullptr, nullptr);
+    }
+    for (long long t = tid; t < ng; t += NT) cur[t] = nk - 1;
+    __syncthreads();
+
+    // ---- G = 2 H e and the starting loss (lines 8-9) ----
+    const double* e0 = R + (size_t)(nk - 1) * d_in;
+    double loss = 0.0;
+    if (VERIFY) {
+      for (long long pp = tid; pp < d_in; pp += NT) {
+        const float* row = p.H + pp * d_in;
+        double acc = 0.0;
+        for (long long k = 0; k < d_in; ++k) acc = __dadd_rn(acc, __dmul_rn((double)row[k], e0[k]));
+        M[pp] = acc;
+        G[pp] = __dmul_rn(2.0, acc);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        double l = 0.0;
+        for (long long pp = 0; pp < d_in; ++pp) l = __dadd_rn(l, __dmul_rn(e0[pp], M[pp]));
+        s_val[0] = l;
+      }
+      __syncthreads();
+      loss = s_val[0];
+      __syncthreads();
+    } else {
+      double part = 0.0;
+      for (long long pp = warp; pp < d_in; pp += nwarps) {
+        const float* row = p.H + pp * d_in;
+        double acc = 0.0;
+        for (long long k = lane; k < d_in; k += 32) acc = fma((double)row[k], e0[k], acc);
+        acc = warp_sum(acc);
+        if (lane == 0) { G[pp] = 2.0 * acc; part = fma(e0[pp], acc, part); }
+      }
+      s_val[tid] = part;
+      __syncthreads();
+      for (int w = NT / 2; w > 0; w >>= 1) {
+        if (tid < w) s_val[tid] += s_val[tid + w];
+        __syncthreads();
+      }
+      loss = s_val[0];
+      __syncthreads();
+      // M(k) = H_tt r(t, k) for every group and grid point: one thread per (k, i)
+      for (long long idx = tid; idx < (long long)nk * d_in; idx += NT) {
+        const int k = (int)(idx / d_in);
+        const long long i = idx - (long long)k * d_in, t0 = (i / g) * g;
+        const float* row = p.H + i * d_in + t0;
+        const double* r = R + (size_t)k * d_in + t0;
+        double acc = 0.0;
+        for (long long q = 0; q < g; ++q) acc = fma((double)row[q], r[q], acc);
+        M[idx] = acc;
+      }
+      __syncthreads();
+    }
+    if (tid == 0) p.col_before[j] = loss;
+
+    // ---- descent over the strengths (lines 10-14) ----
+    const long long ntask = ng * nk;
+    long long nmoves = 0;
+    for (long long step = 0; step < p.steps; ++step) {
+      // score of every (group, grid point); the current point scores +0 and is never taken
+      if (VERIFY) {
+        for (long long task = tid; task < ntask; task += NT) {
+          const long long t = task / nk;
+          const int k = (int)(task - t * nk), c = cur[t];
+          double change = 0.0;
+          if (k != c) {
+            const double* cand = R + (size_t)k * d_in + t * g;
+            const double* old = R + (size_t)c * d_in + t * g;
+            double quad = 0.0, lin = 0.0;
+            for (long long pp = 0; pp < g; ++pp) {
+              const float* row = p.H + (t * g + pp) * d_in + t * g;
+              double acc = 0.0;
+              for (long long r = 0; r < g; ++r)
+                acc = __dadd_rn(acc, __dmul_rn((double)row[r], __dadd_rn(cand[r], -old[r])));
+              const double dp = __dadd_rn(cand[pp], -old[pp]);
+              quad = __dadd_rn(quad, __dmul_rn(dp, acc));
+              lin = __dadd_rn(lin, __dmul_rn(dp, G[t * g + pp]));
+            }
+            change = __dadd_rn(quad, lin);
+          }
+          S[task] = change;
+        }
+      } else {
+        for (long long task = warp; task < ntask; task += nwarps) {
+          const long long t = task / nk;
+          const int k = (int)(task - t * nk), c = cur[t];
+          double v = 0.0;
+          if (k != c) {
+            const double* rk = R + (size_t)k * d_in + t * g;
+            const double* rc = R + (size_t)c * d_in + t * g;
+            const double* mk = M + (size_t)k * d_in + t * g;
+            const double* mc = M + (size_t)c * d_in + t * g;
+            const double* gt = G + t * g;
+            for (long long pp = lane; pp < g; pp += 32) {
+              const double a = rk[pp], b = rc[pp];
+              // delta^T H delta = r_k.M_k - 2 r_k.M_c + r_c.M_c ; delta^T G
+              v += a * mk[pp] - 2.0 * a * mc[pp] + b * mc[pp] + (a - b) * gt[pp];
+            }
+            v = warp_sum(v);
+          }
+          if (lane == 0) S[task] = v;
+        }
+      }
+      __syncthreads();
+      // argmin: lowest (group, grid index) among equal scores
+      double bv = 0.0;
+      int bi = -1;
+      for (long long task = tid; task < ntask; task += NT) {
+        const double v = S[task];
+        if (v < bv) { bv = v; bi = (int)task; }
+      }
+      s_val[tid] = bv; s_idx[tid] = bi;
+      __syncthreads();
+      for (int w = NT / 2; w > 0; w >>= 1) {
+        if (tid < w) {
+          const double ov = s_val[tid + w];
+          const int oi = s_idx[tid + w];
+          const bool take = oi >= 0 && (s_idx[tid] < 0 || ov < s_val[tid] || (ov == s_val[tid] && oi < s_idx[tid]));
+          if (take) { s_val[tid] = ov; s_idx[tid] = oi; }
+        }
+        __syncthreads();
+      }
+      const int best = s_idx[0];
+      const double bchange = s_val[0];
+      __syncthreads();
+      if (best < 0) break;
+      const long long ts = best / nk;
+      const int ks = best - (int)ts * nk, cs = cur[ts];
+      // delta of the winning group, then G <- G + 2 H[:, group] delta
+      for (long long r = tid; r < g; r += NT) S[r] = __dadd_rn(R[(size_t)ks * d_in + ts * g + r], -R[(size_t)cs * d_in + ts * g + r]);
+      __syncthreads();
+      if (VERIFY) {
+        for (long long i = tid; i < d_in; i += NT) {
+          const float* row = p.H + i * d_in + ts * g;
+          double acc = 0.0;
+          for (long long r = 0; r < g; ++r) acc = __dadd_rn(acc, __dmul_rn((double)row[r], S[r]));
+          G[i] = __dadd_rn(G[i], __dmul_rn(2.0, acc));
+        }
+      } else {
+        for (long long i = warp; i < d_in; i += nwarps) {
+          const float* row = p.H + i * d_in + ts * g;
+          double acc = 0.0;
+          for (long long r = lane; r < g; r += 32) acc = fma((double)row[r], S[r], acc);
+          acc = warp_sum(acc);
+          if (lane == 0) G[i] += 2.0 * acc;
+        }
+      }
+      __syncthreads();
+      if (tid == 0) cur[ts] = ks;
+      loss = __dadd_rn(loss, bchange);
+      ++nmoves;
+      __syncthreads();
+    }
+    if (tid == 0) { p.col_after[j] = loss; my_moves += (unsigned long long)nmoves; }
+
+    // ---- emit grid, codes and strengths of the chosen points ----
+    for (long long t = tid; t < ng; t += NT) {
+      float a32;
+      resid(0.0, (double)p.mn[t * p.d_out + j], (double)p.mx[t * p.d_out + j], p.gammas[cur[t]], p.L, &a32, nullptr);
+      p.scale[t * p.d_out + j] = a32;
+      p.zero[t * p.d_out + j] = p.mn[t * p.d_out + j];
+      if (p.gamma_out) p.gamma_out[t * p.d_out + j] = (float)p.gammas[cur[t]];
+    }
+    for (long long i = tid; i < d_in; i += NT) {
+      const long long t = i / g;
+      unsigned char q;
+      resid(load_w(p.W, p.wt, i * p.ldw + j), (double)p.mn[t * p.d_out + j], (double)p.mx[t * p.d_out + j],
+            p.gammas[cur[t]], p.L, nullptr, &q);
+      p.Q[i * p.d_out + j] = q;
+    }
+  }
+  if (tid == 0 && my_moves) atomicAdd(&p.ctr->moves, my_moves);
+}
+
+}  // namespace owc
+
+// ---------------------------------------------------------------------------------------------
+constexpr int kOwcMaxCtas = 296;
+
+struct OwcWs {
+  size_t pmn, pmx, mn, mx, gammas, scratch, cur, col_before, col_after, sums, ctr, total;
+  size_t scratch_per_cta;   // doubles
+  long long cpg;
+};
+static OwcWs owc_ws_layout(long long d_in, long long d_out, long long g, int nk) {
+  OwcWs w{};
+  const long long ng = d_in / g;
+  w.cpg = (g + 255) / 256;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  w.pmn = take(sizeof(float) * ng * w.cpg * d_out);
+  w.pmx = take(sizeof(float) * ng * w.cpg * d_out);
+  w.mn = take(sizeof(float) * ng * d_out);
+  w.mx = take(sizeof(float) * ng * d_out);
+  w.gammas = take(sizeof(double) * nk);
+  const size_t tail = (size_t)(ng * nk > g ? ng * nk : g);
+  w.scratch_per_cta = (2 * (size_t)nk * d_in + (size_t)d_in + tail + 31) / 32 * 32;
+  const long long ctas = d_out < kOwcMaxCtas ? d_out : kOwcMaxCtas;
+  w.scratch = take(sizeof(double) * w.scratch_per_cta * ctas);
+  w.cur = take(sizeof(int) * ng * ctas);
+  w.col_before = take(sizeof(double) * d_out);
+  w.col_after = take(sizeof(double) * d_out);
+  w.sums = take(sizeof(double) * 2);
+  w.ctr = take(sizeof(owc::Counters));
+  w.total = off;
+  return w;
+}
+
+size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip) {
+  return owc_ws_layout(d_in, d_out, g, n_clip).total;
+}
+
+// Enqueues the whole OWC-CD on `st`.  host_moves / host_before / host_after (all NULL or all
+// non-NULL) are filled after a stream synchronisation.
+cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long steps, float* scale, float* zero,
+                          unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws, unsigned long long* host_moves,
+                          double* host_before, double* host_after, cudaStream_t st) {
+  const long long d_in = ly.d_in, d_out = ly.d_out, g = ly.g, ng = ly.ng;
+  const int nk = grid.n_clip;
+  const OwcWs L = owc_ws_layout(d_in, d_out, g, nk);
+  char* base = (char*)ws;
+  float* mn = (float*)(base + L.mn);
+  float* mx = (float*)(base + L.mx);
+  cudaError_t e = launch_group_minmax(ly, (float*)(base + L.pmn), (float*)(base + L.pmx), mn, mx, st);
+  if (e != cudaSuccess) return e;
+  double hg[256];
+  const double lo = (double)grid.clip_lo, hi = (double)grid.clip_hi;
+  for (int k = 0; k < nk; ++k) hg[k] = nk > 1 ? lo + ((hi - lo) * (double)k) / (double)(nk - 1) : 1.0;
+  e = cudaMemcpyAsync(base + L.gammas, hg, sizeof(double) * nk, cudaMemcpyHostToDevice, st);  // pageable: staged before return
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(base + L.ctr, 0, sizeof(owc::Counters), st);
+  if (e != cudaSuccess) return e;
+
+  owc::Params p{};
+  p.H = ly.H; p.W = ly.W; p.wt = ly.wt; p.d_in = d_in; p.d_out = d_out; p.ldw = ly.ldw; p.g = g; p.ng = ng;
+  p.L = ly.L; p.nk = nk; p.gammas = (const double*)(base + L.gammas); p.mn = mn; p.mx = mx; p.steps = steps;
+  p.scale = scale; p.zero = zero; p.Q = Q; p.gamma_out = gamma_out;
+  p.scratch = (double*)(base + L.scratch); p.scratch_per_cta = L.scratch_per_cta; p.cur = (int*)(base + L.cur);
+  p.col_before = (double*)(base + L.col_before); p.col_after = (double*)(base + L.col_after);
+  p.ctr = (owc::Counters*)(base + L.ctr);
+  const unsigned ctas = (unsigned)(d_out < kOwcMaxCtas ? d_out : kOwcMaxCtas);
+  if (mode == CDQ_MODE_FP64_VERIFY) owc::owc_cd_kernel<true><<<ctas, owc::NT, 0, st>>>(p);
+  else owc::owc_cd_kernel<false><<<ctas, owc::NT, 0, st>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (host_moves) {
+    double* sums = (double*)(base + L.sums);
+    e = launch_sum_f64(p.col_before, d_out, sums, st);
+    if (e != cudaSuccess) return e;
+    e = launch_sum_f64(p.col_after, d_out, sums + 1, st);
+    if (e != cudaSuccess) return e;
+    owc::Counters hc;
+    double hs[2];
+    e = cudaMemcpyAsync(&hc, p.ctr, sizeof(hc), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return e;
+    e = cudaMemcpyAsync(hs, sums, sizeof(hs), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return e;
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return e;
+    *host_moves = hc.moves; *host_before = hs[0]; *host_after = hs[1];
+  }
+  return cudaSuccess;
+}
+
+}  // namespace cdq
