@@ -160,6 +160,9 @@ def main():
     ap.add_argument("--config", default="C1", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--init", default="rtn", choices=["rtn", "owc_cd"],
+                    help="grid stage: cdq_init_rtn (MinMax / OWC as the config says) or cdq_init_owc_cd (Algorithm 3; "
+                         "configs with a clipping grid)")
     ap.add_argument("--d-out", type=int, default=0, help="profiling case: keep only this many output columns")
     ap.add_argument("--n", type=int, default=0, help="profiling case: keep only this many calibration rows")
     args = ap.parse_args()
@@ -170,8 +173,11 @@ def main():
     cfg = inputs.CONFIGS[args.config]
     if args.d_out or args.n:
         cfg = cfg.scaled(d_out=args.d_out or cfg.d_out, n=args.n or cfg.n)
+    if args.init == "owc_cd" and cfg.n_clip < 2:
+        ap.error("--init owc_cd needs a config with a clipping grid (C2, C4)")
     workload = (f"{cfg.name}: d_in={cfg.d_in} d_out={cfg.d_out} n={cfg.n} X={cfg.x_dtype} W={cfg.w_dtype} "
-                f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}")
+                f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}"
+                + (" init=OWC-CD" if args.init == "owc_cd" else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -210,7 +216,10 @@ def main():
         ev[1].record()
         H = B.cdq_hessian(Xd, ws=ws)
         ev[2].record()
-        scale, zero, Q, _ = B.cdq_init_rtn(Wd, grid, H=H if cfg.n_clip > 1 else None, ws=ws)
+        if args.init == "owc_cd":
+            scale, zero, Q, _, _ = B.cdq_init_owc_cd(Wd, grid, H, ws=ws)
+        else:
+            scale, zero, Q, _ = B.cdq_init_rtn(Wd, grid, H=H if cfg.n_clip > 1 else None, ws=ws)
         ev[3].record()
         stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws)
         ev[4].record()

@@ -193,7 +193,7 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
       if (!grid || d_out < 1 || grid->n_clip < 2 || grid->n_clip > 256) return 0;
       const long long g = grid->group_size > 0 ? grid->group_size : d_in;
       if (g < 1 || d_in % g) return 0;
-      return owc_cd_workspace(d_in, d_out, g, grid->n_clip);
+      return owc_cd_workspace(d_in, d_out, g, grid->n_clip, mode);
     }
     case CDQ_CALL_CD_SOLVE:
       if (d_out < 1) return 0;
@@ -258,7 +258,7 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
   if (grid->n_clip < 2) return CDQ_ERR_INVALID_ARG;
   Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, nullptr, nullptr);
   if (ly.ng > 65535) return CDQ_ERR_UNSUPPORTED;
-  s = check_ws(ws, ws_bytes, owc_cd_workspace(d_in, d_out, ly.g, grid->n_clip));
+  s = check_ws(ws, ws_bytes, owc_cd_workspace(d_in, d_out, ly.g, grid->n_clip, mode));
   if (s != CDQ_OK) return s;
   if (steps <= 0) steps = ly.ng;
   unsigned long long moves = 0;

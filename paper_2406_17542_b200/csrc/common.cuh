@@ -62,7 +62,7 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
 cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* mn, float* mx, cudaStream_t st);
 
 // owc_cd.cu : greedy descent over per-group clipping strengths (paper: Algorithm 3)
-size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip);
+size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip, cdq_mode mode);
 cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long steps, float* scale, float* zero,
                           unsigned char* Q, float* gamma_out, cdq_mode mode, void* ws, unsigned long long* host_moves,
                           double* host_before, double* host_after, cudaStream_t st);

@@ -23,7 +23,8 @@
 namespace cdq {
 namespace owc {
 
-constexpr int NT = 256;
+constexpr int NT = 512;
+constexpr int KC = 8;     // grid points per pass of the M table (accumulators per thread)
 
 struct Counters {
   int next_col;
@@ -50,6 +51,8 @@ struct Params {
   int* cur;               // per CTA: [ng]
   double* col_before;     // [d_out]
   double* col_after;      // [d_out]
+  double* Gext;           // FAST, optional: [d_out, ldg] G = 2 H e at the start, made by the tensor-core GEMM
+  long long ldg;          //   (then col_before is already filled and the kernel skips that product)
   Counters* ctr;
 };
 
@@ -77,17 +80,18 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 template <bool VERIFY>
-__global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
+__global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
   __shared__ int s_col;
   __shared__ double s_val[NT];
   __shared__ int s_idx[NT];
+  extern __shared__ double dyn[];   // FAST: quad [ng * nk] (delta^T H_tt delta per candidate), rg [ng * nk] (r_k . G_t)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
   const long long d_in = p.d_in, g = p.g, ng = p.ng;
   const int nk = p.nk;
   double* R = p.scratch + (size_t)blockIdx.x * p.scratch_per_cta;   // [nk, d_in] residuals
   double* M = R + (size_t)nk * d_in;                                 // [nk, d_in] H_tt r (FAST), H e (VERIFY, row 0)
-  double* G = M + (size_t)nk * d_in;                                 // [d_in]
-  double* S = G + d_in;                                              // [max(ng * nk, g)] scores / delta
+  double* Gown = M + (size_t)nk * d_in;                              // [d_in]
+  double* S = Gown + d_in;                                            // [max(ng * nk, g)] scores / delta
   int* cur = p.cur + (size_t)blockIdx.x * ng;
   unsigned long long my_moves = 0;
 
@@ -109,6 +113,7 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
     __syncthreads();
 
     // ---- G = 2 H e and the starting loss (lines 8-9) ----
+    double* G = (!VERIFY && p.Gext) ? p.Gext + j * p.ldg : Gown;
     const double* e0 = R + (size_t)(nk - 1) * d_in;
     double loss = 0.0;
     if (VERIFY) {
@@ -129,39 +134,87 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
       loss = s_val[0];
       __syncthreads();
     } else {
-      double part = 0.0;
-      for (long long pp = warp; pp < d_in; pp += nwarps) {
-        const float* row = p.H + pp * d_in;
-        double acc = 0.0;
-        for (long long k = lane; k < d_in; k += 32) acc = fma((double)row[k], e0[k], acc);
-        acc = warp_sum(acc);
-        if (lane == 0) { G[pp] = 2.0 * acc; part = fma(e0[pp], acc, part); }
-      }
-      s_val[tid] = part;
-      __syncthreads();
-      for (int w = NT / 2; w > 0; w >>= 1) {
-        if (tid < w) s_val[tid] += s_val[tid + w];
+      if (p.Gext) {
+        loss = p.col_before[j];
+      } else {
+        double part = 0.0;
+        for (long long pp = warp; pp < d_in; pp += nwarps) {
+          const float* row = p.H + pp * d_in;
+          double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+          long long k = lane;
+          for (; k + 96 < d_in; k += 128) {
+            a0 = fma((double)row[k], e0[k], a0);
+            a1 = fma((double)row[k + 32], e0[k + 32], a1);
+            a2 = fma((double)row[k + 64], e0[k + 64], a2);
+            a3 = fma((double)row[k + 96], e0[k + 96], a3);
+          }
+          for (; k < d_in; k += 32) a0 = fma((double)row[k], e0[k], a0);
+          const double acc = warp_sum((a0 + a1) + (a2 + a3));
+          if (lane == 0) { G[pp] = 2.0 * acc; part = fma(e0[pp], acc, part); }
+        }
+        s_val[tid] = part;
+        __syncthreads();
+        for (int w = NT / 2; w > 0; w >>= 1) {
+          if (tid < w) s_val[tid] += s_val[tid + w];
+          __syncthreads();
+        }
+        loss = s_val[0];
         __syncthreads();
       }
-      loss = s_val[0];
-      __syncthreads();
-      // M(k) = H_tt r(t, k) for every group and grid point: one thread per (k, i)
-      for (long long idx = tid; idx < (long long)nk * d_in; idx += NT) {
-        const int k = (int)(idx / d_in);
-        const long long i = idx - (long long)k * d_in, t0 = (i / g) * g;
+      // M(k) = H_tt r(t, k): one thread per coordinate i and pass of KC grid points, so that a
+      // value of H feeds KC independent accumulators
+      const int npass = (nk + KC - 1) / KC;
+      for (long long idx = tid; idx < (long long)npass * d_in; idx += NT) {
+        const int ps = (int)(idx / d_in);
+        const long long i = idx - (long long)ps * d_in, t0 = (i / g) * g;
         const float* row = p.H + i * d_in + t0;
-        const double* r = R + (size_t)k * d_in + t0;
-        double acc = 0.0;
-        for (long long q = 0; q < g; ++q) acc = fma((double)row[q], r[q], acc);
-        M[idx] = acc;
+        double acc[KC];
+#pragma unroll
+        for (int c = 0; c < KC; ++c) acc[c] = 0.0;
+#pragma unroll 4
+        for (long long q = 0; q < g; ++q) {
+          const double h = (double)row[q];
+#pragma unroll
+          for (int c = 0; c < KC; ++c) {
+            const int k = ps * KC + c;
+            if (k < nk) acc[c] = fma(h, R[(size_t)k * d_in + t0 + q], acc[c]);
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < KC; ++c) {
+          const int k = ps * KC + c;
+          if (k < nk) M[(size_t)k * d_in + i] = acc[c];
+        }
       }
       __syncthreads();
     }
-    if (tid == 0) p.col_before[j] = loss;
+    if (tid == 0 && (VERIFY || !p.Gext)) p.col_before[j] = loss;
 
     // ---- descent over the strengths (lines 10-14) ----
     const long long ntask = ng * nk;
     long long nmoves = 0;
+    double* quad_s = dyn;
+    double* rg_s = dyn + ntask;
+    // delta^T H_tt delta = r_k.M_k - 2 r_k.M_c + r_c.M_c for every candidate of the groups [t_lo, t_hi)
+    auto refresh_quad = [&](long long t_lo, long long t_hi) {
+      for (long long task = t_lo * nk + warp; task < t_hi * nk; task += nwarps) {
+        const long long t = task / nk;
+        const int k = (int)(task - t * nk), c = cur[t];
+        const double* rk = R + (size_t)k * d_in + t * g;
+        const double* rc = R + (size_t)c * d_in + t * g;
+        const double* mk = M + (size_t)k * d_in + t * g;
+        const double* mc = M + (size_t)c * d_in + t * g;
+        double v = 0.0;
+#pragma unroll 4
+        for (long long pp = lane; pp < g; pp += 32) {
+          const double a = rk[pp], b = rc[pp], m = mc[pp];
+          v += a * mk[pp] - 2.0 * a * m + b * m;
+        }
+        v = warp_sum(v);
+        if (lane == 0) quad_s[task] = v;
+      }
+    };
+    if (!VERIFY) { refresh_quad(0, ng); __syncthreads(); }
     for (long long step = 0; step < p.steps; ++step) {
       // score of every (group, grid point); the current point scores +0 and is never taken
       if (VERIFY) {
@@ -187,24 +240,29 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
           S[task] = change;
         }
       } else {
-        for (long long task = warp; task < ntask; task += nwarps) {
+        // r_k . G_t for every candidate: one warp per group and four grid points, so that 16 loads are in flight
+        const int kq = (nk + 3) / 4;
+        for (long long wt = warp; wt < ng * kq; wt += nwarps) {
+          const long long t = wt / kq;
+          const int k0 = (int)(wt - t * kq) * 4;
+          double acc[4] = {0.0, 0.0, 0.0, 0.0};
+          for (long long pp = lane; pp < g; pp += 32) {
+            const double gv = G[t * g + pp];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              if (k0 + u < nk) acc[u] = fma(R[(size_t)(k0 + u) * d_in + t * g + pp], gv, acc[u]);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const double a = warp_sum(acc[u]);
+            if (lane == 0 && k0 + u < nk) rg_s[t * nk + k0 + u] = a;
+          }
+        }
+        __syncthreads();
+        for (long long task = tid; task < ntask; task += NT) {
           const long long t = task / nk;
           const int k = (int)(task - t * nk), c = cur[t];
-          double v = 0.0;
-          if (k != c) {
-            const double* rk = R + (size_t)k * d_in + t * g;
-            const double* rc = R + (size_t)c * d_in + t * g;
-            const double* mk = M + (size_t)k * d_in + t * g;
-            const double* mc = M + (size_t)c * d_in + t * g;
-            const double* gt = G + t * g;
-            for (long long pp = lane; pp < g; pp += 32) {
-              const double a = rk[pp], b = rc[pp];
-              // delta^T H delta = r_k.M_k - 2 r_k.M_c + r_c.M_c ; delta^T G
-              v += a * mk[pp] - 2.0 * a * mc[pp] + b * mc[pp] + (a - b) * gt[pp];
-            }
-            v = warp_sum(v);
-          }
-          if (lane == 0) S[task] = v;
+          S[task] = k == c ? 0.0 : quad_s[task] + (rg_s[task] - rg_s[t * nk + c]);
         }
       }
       __syncthreads();
@@ -243,12 +301,23 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
           G[i] = __dadd_rn(G[i], __dmul_rn(2.0, acc));
         }
       } else {
-        for (long long i = warp; i < d_in; i += nwarps) {
+        // one thread per row: 4 independent accumulators over the group's g columns (a warp per row
+        // would spend more instructions on the shuffle reduction than on the g / 32 products per lane)
+        for (long long i = tid; i < d_in; i += NT) {
           const float* row = p.H + i * d_in + ts * g;
-          double acc = 0.0;
-          for (long long r = lane; r < g; r += 32) acc = fma((double)row[r], S[r], acc);
-          acc = warp_sum(acc);
-          if (lane == 0) G[i] += 2.0 * acc;
+          double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+          long long r = 0;
+          if ((g & 3) == 0 && ((reinterpret_cast<uintptr_t>(row) & 15) == 0)) {
+            for (; r < g; r += 4) {
+              const float4 h = *reinterpret_cast<const float4*>(row + r);
+              a0 = fma((double)h.x, S[r], a0);
+              a1 = fma((double)h.y, S[r + 1], a1);
+              a2 = fma((double)h.z, S[r + 2], a2);
+              a3 = fma((double)h.w, S[r + 3], a3);
+            }
+          }
+          for (; r < g; ++r) a0 = fma((double)row[r], S[r], a0);
+          G[i] += 2.0 * ((a0 + a1) + (a2 + a3));
         }
       }
       __syncthreads();
@@ -256,6 +325,7 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
       loss = __dadd_rn(loss, bchange);
       ++nmoves;
       __syncthreads();
+      if (!VERIFY) { refresh_quad(ts, ts + 1); __syncthreads(); }
     }
     if (tid == 0) { p.col_after[j] = loss; my_moves += (unsigned long long)nmoves; }
 
@@ -284,11 +354,13 @@ __global__ void __launch_bounds__(NT) owc_cd_kernel(Params p) {
 constexpr int kOwcMaxCtas = 296;
 
 struct OwcWs {
-  size_t pmn, pmx, mn, mx, gammas, scratch, cur, col_before, col_after, sums, ctr, total;
+  size_t pmn, pmx, mn, mx, gammas, scratch, cur, col_before, col_after, sums, ctr, E, G, hbuf, ebuf, total;
+  bool tc;            // starting gradient by the int8 tensor-core GEMM (production mode, large enough layers)
+  long long ldg;
   size_t scratch_per_cta;   // doubles
   long long cpg;
 };
-static OwcWs owc_ws_layout(long long d_in, long long d_out, long long g, int nk) {
+static OwcWs owc_ws_layout(long long d_in, long long d_out, long long g, int nk, cdq_mode mode) {
   OwcWs w{};
   const long long ng = d_in / g;
   w.cpg = (g + 255) / 256;
@@ -308,12 +380,20 @@ static OwcWs owc_ws_layout(long long d_in, long long d_out, long long g, int nk)
   w.col_after = take(sizeof(double) * d_out);
   w.sums = take(sizeof(double) * 2);
   w.ctr = take(sizeof(owc::Counters));
+  w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+  w.ldg = (d_in + 3) / 4 * 4;
+  if (w.tc) {
+    w.E = take(sizeof(double) * d_in * d_out);
+    w.G = take(sizeof(double) * d_out * w.ldg);
+    w.hbuf = take(gemm_tc_h_bytes(d_in, kTcGradNH));
+    w.ebuf = take(gemm_tc_e_bytes(d_in, d_out, kTcGradNE));
+  }
   w.total = off;
   return w;
 }
 
-size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip) {
-  return owc_ws_layout(d_in, d_out, g, n_clip).total;
+size_t owc_cd_workspace(long long d_in, long long d_out, long long g, int n_clip, cdq_mode mode) {
+  return owc_ws_layout(d_in, d_out, g, n_clip, mode).total;
 }
 
 // Enqueues the whole OWC-CD on `st`.  host_moves / host_before / host_after (all NULL or all
@@ -323,7 +403,7 @@ cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long 
                           double* host_before, double* host_after, cudaStream_t st) {
   const long long d_in = ly.d_in, d_out = ly.d_out, g = ly.g, ng = ly.ng;
   const int nk = grid.n_clip;
-  const OwcWs L = owc_ws_layout(d_in, d_out, g, nk);
+  const OwcWs L = owc_ws_layout(d_in, d_out, g, nk, mode);
   char* base = (char*)ws;
   float* mn = (float*)(base + L.mn);
   float* mx = (float*)(base + L.mx);
@@ -344,9 +424,34 @@ cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long 
   p.scratch = (double*)(base + L.scratch); p.scratch_per_cta = L.scratch_per_cta; p.cur = (int*)(base + L.cur);
   p.col_before = (double*)(base + L.col_before); p.col_after = (double*)(base + L.col_after);
   p.ctr = (owc::Counters*)(base + L.ctr);
+  if (L.tc) {   // G = 2 H e and the column losses at the starting strengths
+    ResidualSrc src{};
+    src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw; src.mn = mn; src.mx = mx; src.gamma = hg[nk - 1]; src.L = ly.L;
+    src.use_gamma = 1; src.g = g; src.d_out = d_out;
+    double* E = (double*)(base + L.E);
+    e = launch_residual_f64(src, d_in, E, st);
+    if (e != cudaSuccess) return e;
+    e = gemm_tc_prepare_h(ly.H, d_in, kTcGradNH, base + L.hbuf, st);
+    if (e != cudaSuccess) return e;
+    p.Gext = (double*)(base + L.G); p.ldg = L.ldg;
+    e = gemm_tc_run(base + L.hbuf, kTcGradNH, E, d_in, d_out, kTcGradNE, kTcGradSmax, 2.0, p.Gext, p.ldg, p.col_before,
+                    base + L.ebuf, st);
+    if (e != cudaSuccess) return e;
+  }
   const unsigned ctas = (unsigned)(d_out < kOwcMaxCtas ? d_out : kOwcMaxCtas);
-  if (mode == CDQ_MODE_FP64_VERIFY) owc::owc_cd_kernel<true><<<ctas, owc::NT, 0, st>>>(p);
-  else owc::owc_cd_kernel<false><<<ctas, owc::NT, 0, st>>>(p);
+  // the production kernel keeps two tables of ng * n_clip doubles in shared memory; grids too fine for
+  // that run the fixed-order kernel (slower, same result)
+  const size_t smem = 2 * sizeof(double) * (size_t)ng * nk;
+  if (mode == CDQ_MODE_FP64_VERIFY || smem > 160 * 1024) {
+    p.Gext = nullptr;
+    owc::owc_cd_kernel<true><<<ctas, owc::NT, 0, st>>>(p);
+  } else {
+    if (smem > 40 * 1024) {
+      e = cudaFuncSetAttribute(owc::owc_cd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    owc::owc_cd_kernel<false><<<ctas, owc::NT, smem, st>>>(p);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (host_moves) {
