@@ -160,6 +160,9 @@ def main():
     ap.add_argument("--config", default="C1", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--budget-div", type=int, default=0,
+                    help="descent budget T = d_in / DIV steps per column (the paper's fewer-iterations study) "
+                         "instead of the config's passes * d_in")
     ap.add_argument("--init", default="rtn", choices=["rtn", "owc_cd"],
                     help="grid stage: cdq_init_rtn (MinMax / OWC as the config says) or cdq_init_owc_cd (Algorithm 3; "
                          "configs with a clipping grid)")
@@ -177,7 +180,8 @@ def main():
         ap.error("--init owc_cd needs a config with a clipping grid (C2, C4)")
     workload = (f"{cfg.name}: d_in={cfg.d_in} d_out={cfg.d_out} n={cfg.n} X={cfg.x_dtype} W={cfg.w_dtype} "
                 f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}"
-                + (" init=OWC-CD" if args.init == "owc_cd" else ""))
+                + (" init=OWC-CD" if args.init == "owc_cd" else "")
+                + (f" budget=d_in/{args.budget_div}" if args.budget_div > 0 else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -221,7 +225,8 @@ def main():
         else:
             scale, zero, Q, _ = B.cdq_init_rtn(Wd, grid, H=H if cfg.n_clip > 1 else None, ws=ws)
         ev[3].record()
-        stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws)
+        stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
+                               steps_per_col=cfg.d_in // args.budget_div if args.budget_div > 0 else None)
         ev[4].record()
         loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws)
         if host:

@@ -178,6 +178,17 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
                         cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same descent with the budget given in steps per column instead of passes: T = steps_per_col
+ * (paper: the study of fewer iterations, T = d_in / 2, d_in / 4, d_in / 8, in the appendix on
+ * speeding up CD; Algorithm 1 takes T as its input).  cdq_cd_solve(passes) is
+ * cdq_cd_solve_steps(passes * d_in).
+ */
+cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                              long long ldw, const cdq_grid_desc* grid, const float* scale,
+                              const float* zero, unsigned char* Q, long long steps_per_col, cdq_mode mode,
+                              cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Layer loss sum_j e_j^T H e_j with e = W_hat - W (paper: Eq. 1 written with
  * H = X^T X; the objective value the paper reports for a solution).
  *   loss     host pointer to one double, may be NULL.

@@ -269,10 +269,11 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
   return CDQ_OK;
 }
 
-cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
-                        const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
-                        int passes, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
-  if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || passes < 0)
+static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                                const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
+                                long long steps_per_col, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes,
+                                void* stream) {
+  if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || steps_per_col < 0)
     return CDQ_ERR_INVALID_ARG;
   cdq_status s = check_layer_shape(d_in, d_out, ldw);
   if (s != CDQ_OK) return s;
@@ -293,7 +294,6 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
   double* col_loss = (double*)(base + L.col_loss);
   double* loss_sum = (double*)(base + L.scalars);
   CdCounters* ctr = (CdCounters*)(base + L.scalars + 64);
-  const long long steps_per_col = (long long)passes * d_in;
 
   // G0 = 2 H (W_hat - W) and the loss at entry
   CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
@@ -346,6 +346,22 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
     return read_device_status_after_sync();
   }
   return CDQ_OK;
+}
+
+cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                        const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
+                        int passes, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
+  if (passes < 0) return CDQ_ERR_INVALID_ARG;
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, (long long)passes * d_in, mode, stats, ws,
+                       ws_bytes, stream);
+}
+
+cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                              long long ldw, const cdq_grid_desc* grid, const float* scale, const float* zero,
+                              unsigned char* Q, long long steps_per_col, cdq_mode mode, cdq_cd_stats* stats, void* ws,
+                              size_t ws_bytes, void* stream) {
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, mode, stats, ws, ws_bytes,
+                       stream);
 }
 
 cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,

@@ -166,3 +166,25 @@ def test_hessian_tensor_core_path(n, d_in):
     H2 = B.cdq_hessian(Xd[:half])
     H2 = B.cdq_hessian(Xd[half:], accumulate=True, out=H2)
     assert rel_fro(H2.cpu().numpy(), Hc) <= 1e-5
+
+
+@pytest.mark.parametrize("mode", ["verify", "fast"])
+@pytest.mark.parametrize("frac", [8, 2])
+def test_reduced_step_budget(mode, frac):
+    """T = d_in / 8 and d_in / 2 steps per column (the paper's fewer-iterations study) against the oracle."""
+    cfg = inputs.CONFIGS["C0"]
+    X, W = inputs.make_layer(cfg)
+    _, H32 = oracle.hessian(X)
+    init = oracle.init_rtn(W, cfg.bits, cfg.group_size)
+    T = cfg.d_in // frac
+    ref = oracle.cd_solve(H32, W, cfg.bits, init["scale"], init["zero"], init["Q"], T)
+    Hd = torch.from_numpy(H32).cuda(); Wd = W.cuda()
+    g = grid_of(cfg)
+    scale, zero, Q, _ = B.cdq_init_rtn(Wd, g, mode=mode)
+    st = B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, 0, mode=mode, steps_per_col=T)
+    assert st["steps"] == T * cfg.d_out and st["committed"] <= st["steps"]
+    if mode == "verify":
+        assert np.array_equal(Q.cpu().numpy(), ref["Q"]) and st["committed"] == ref["committed"]
+    else:
+        assert float((Q.cpu().numpy() == ref["Q"]).mean()) >= CODE_AGREE
+        np.testing.assert_allclose(st["loss_after"], ref["loss_after"], rtol=LOSS_RTOL)
