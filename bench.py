@@ -26,7 +26,7 @@ sys.path.insert(0, ROOT)
 
 import torch  # noqa: E402
 
-from paper_2406_17542_b200 import inputs  # noqa: E402
+from paper_2406_17542_b200 import inputs, multi  # noqa: E402
 
 METRIC = "cd_coordinate_updates_per_s"
 UNIT = "updates/s"
@@ -200,7 +200,7 @@ def main():
 
     # every rank quantizes its own layer (same shape, its own seed): columns and layers are
     # independent problems, so there is no data-path collective
-    my_cfg = cfg.scaled(seed=cfg.seed + 1000 * rank)
+    my_cfg = cfg.scaled(seed=multi.rank_seed(cfg.seed, rank))
     X, W = inputs.make_layer(my_cfg, device=dev)
     Xh, Wh = X.cpu().pin_memory(), W.cpu().pin_memory()
     grid = B.Grid(cfg.bits, cfg.group_size, cfg.n_clip, cfg.clip_lo, cfg.clip_hi)
@@ -208,9 +208,7 @@ def main():
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        multi.barrier(world)
 
     def one_step(host: bool, times: dict | None = None):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
@@ -267,15 +265,7 @@ def main():
     total_ms = sum(times["total"])
     total_ms_e2e = sum(times_e2e["total"])
     committed = stats["committed"]
-    if world > 1:
-        t = torch.tensor([total_ms, total_ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, total_ms_e2e = t.tolist()
-        c = torch.tensor([committed], dtype=torch.float64, device=dev)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        committed_all = c.item()
-    else:
-        committed_all = float(committed)
+    (total_ms, total_ms_e2e), committed_all = multi.aggregate([total_ms, total_ms_e2e], committed, world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -283,7 +273,7 @@ def main():
 
     peaks = load_peaks()
     ms_per_step = total_ms / args.steps
-    value = committed_all / (ms_per_step * 1e-3)
+    value = multi.whole_job_throughput(committed_all, total_ms, args.steps)
     mean = lambda v: sum(v) / len(v)
     cd_ms = mean(times["cd_kernel"])
     alg_bytes = algorithmic_bytes_cd(cfg, committed)
