@@ -58,6 +58,10 @@ def _load():
     lib.cdqo_gamma.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double]
     lib.cdqo_hessian.argtypes = [_dp, _i64, _i64, ctypes.c_double, _dp, _fp]
     lib.cdqo_hessian_entries.argtypes = [_dp, _i64, _i64, _i64p, _i64p, _i64, _dp]
+    lib.cdqo_bcd_perm.restype = _i64
+    lib.cdqo_bcd_perm.argtypes = [_i64, _i64, ctypes.c_ulonglong, _i64, _i64]
+    lib.cdqo_bcd_solve.argtypes = [_fp, _dp, _i64, _i64, ctypes.c_int, _i64, _fp, _fp, _u8p, ctypes.c_int, _i64,
+                                   ctypes.c_ulonglong, _i64p, _dp, _dp]
     lib.cdqo_owc_cd.argtypes = [_dp, _i64, _i64, _fp, ctypes.c_int, _i64, ctypes.c_int, ctypes.c_double,
                                 ctypes.c_double, _i64, _fp, _fp, _u8p, _ip, _i64p, _dp, _dp]
     lib.cdqo_init_rtn.argtypes = [_dp, _i64, _i64, _fp, ctypes.c_int, _i64, ctypes.c_int,
@@ -176,6 +180,27 @@ def owc_cd(H, W, bits: int, group_size: int, n_clip: int, clip_lo: float, clip_h
     assert rc == 0, rc
     return {"scale": scale, "zero": zero, "Q": Q, "gamma_idx": gidx, "moves": moves,
             "loss_before": lb, "loss_after": la}
+
+
+def bcd_perm(d_in: int, seed: int, col: int, step: int) -> np.ndarray:
+    """The pseudo-random permutation pi that cuts the coordinates into blocks at one step of one column."""
+    lib = _load()
+    return np.array([lib.cdqo_bcd_perm(x, d_in, seed, col, step) for x in range(d_in)], dtype=np.int64)
+
+
+def bcd_solve(H, W, bits: int, scale, zero, Q, k: int, steps_per_col: int, seed: int = 0, group_size: int = 0) -> dict:
+    """Block coordinate descent with random blocks of size k (Algorithm 2 / Algorithm 5), from the codes Q."""
+    Hf, W, scale, zero = _f32(H), _f64(W), _f32(scale), _f32(zero)
+    Q = np.array(_u8(Q), copy=True)
+    d_in, d_out = W.shape
+    moves = np.zeros(d_out, dtype=np.int64)
+    lb = np.zeros(d_out, dtype=np.float64)
+    la = np.zeros(d_out, dtype=np.float64)
+    rc = _load().cdqo_bcd_solve(_ptr(Hf, _fp), _ptr(W, _dp), d_in, d_out, int(bits), int(group_size), _ptr(scale, _fp),
+                                _ptr(zero, _fp), _ptr(Q, _u8p), int(k), int(steps_per_col), int(seed),
+                                _ptr(moves, _i64p), _ptr(lb, _dp), _ptr(la, _dp))
+    assert rc == 0, rc
+    return {"Q": Q, "moves": moves, "loss_before": lb, "loss_after": la}
 
 
 def gradient(H, W, scale, zero, Q, group_size: int = 0) -> np.ndarray:

@@ -17,6 +17,8 @@
  *   - the layer loss  sum_j e_j^T H e_j            (Eq. 1 written with H)
  *   - OWC-CD: greedy descent over per-group clipping strengths (Algorithm 3;
  *     its readings are listed above cdqo_owc_cd)
+ *   - BCD with random blocks (Algorithm 2 / Algorithm 5; readings above
+ *     cdqo_bcd_solve, including the counter-based partition)
  *
  * Formulation.  Algorithm 1 works in code units (g = 2H(q - (w-b)/a), the
  * printed decrease (r-q_i)^2 H_ii + (r-q_i) g_i is the loss change divided by
@@ -53,6 +55,10 @@
  * tracked loss against the loss recomputed from X; one group == the OWC grid
  * search; brute force over all assignments of grid points to groups; first
  * change == best single-group change; convergence == no improving change.
+ * BCD: the partition is a permutation that varies with step, column and seed
+ * and reaches every pair; block size 1 == the greedy descent; one step == the
+ * brute-force best block move with the loss from the definition; prefixes of
+ * a run are monotone.
  * Parity unpinned: anything that depends on the paper's (unstated) lambda.
  */
 #include <math.h>
@@ -569,6 +575,152 @@ int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
       if (loss_after) loss_after[j] = loss;
     }
     free(w); free(tab); free(G); free(e); free(he); free(delta); free(q); free(a); free(b); free(cur);
+  }
+  return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* BCD with random blocks (Algorithm 2; Algorithm 5 for sub-channel grids),  */
+/* block size k, weight-unit form as for the greedy descent above.           */
+/*                                                                           */
+/* Step t of column j: the coordinates are cut into d_in / k blocks by a     */
+/* pseudo-random permutation pi (block u = {pi(k u), ..., pi(k u + k - 1)}); */
+/* for every block and every assignment r of levels to its coordinates, with */
+/* d_i = a_i (r_i - q_i),                                                    */
+/*     change = sum_i d_i^2 H_ii + 2 sum_{i<m} d_i d_m H_im + sum_i d_i G_i  */
+/* (line 6: (r-q)^T H_bb (r-q) + (r-q)^T g_b in weight units); the most      */
+/* negative change is applied: q_b <- r, G <- G + 2 sum_i d_i H[i, :].       */
+/*                                                                           */
+/* Readings:                                                                 */
+/*  - the partition (line 5 says only "randomly partition"): pi is a         */
+/*    counter-based bijection of {0..d_in-1}, the same on every              */
+/*    implementation: with b = bits of d_in - 1 and mask = 2^b - 1, three    */
+/*    rounds  x <- (x * (2 K_r + 1) + (K_r >> 33)) & mask;  x <- x ^ (x >> s) */
+/*    with                                                                   */
+/*    s = max(1, b / 2) and K_r = splitmix64(seed, j, t, r) (each round is a */
+/*    bijection of b-bit words), repeated while x >= d_in (cycle walking).   */
+/*    splitmix64 is the published finaliser  z += 0x9E3779B97F4A7C15;        */
+/*    z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9; z = (z ^ z >> 27) *            */
+/*    0x94D049BB133111EB; z ^ z >> 31  applied to                            */
+/*    seed ^ (j << 40) ^ (t << 8) ^ r folded as below;                       */
+/*  - a step whose partition holds no improving block changes nothing and    */
+/*    the next step draws the next partition (the loop does not stop);       */
+/*  - ties: the block whose smallest coordinate is lowest, then the          */
+/*    assignment that is lowest in the order of the block's coordinates      */
+/*    sorted ascending; for k = 1 this is the rule of the greedy descent,    */
+/*    which BCD then reproduces exactly.                                     */
+/* ------------------------------------------------------------------------ */
+static unsigned long long cdqo_splitmix64(unsigned long long z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+/* keys of the three rounds for (seed, column, step) */
+static void bcd_round_keys(unsigned long long seed, i64 j, i64 t, unsigned long long key[3]) {
+  const unsigned long long base = cdqo_splitmix64(seed ^ cdqo_splitmix64((unsigned long long)j));
+  for (int r = 0; r < 3; ++r) key[r] = cdqo_splitmix64(base ^ (((unsigned long long)t << 2) | (unsigned long long)r));
+}
+/* pi(x) for the partition of step t; exported for the tests */
+i64 cdqo_bcd_perm(i64 x, i64 d_in, unsigned long long seed, i64 j, i64 t) {
+  int b = 0;
+  while (((i64)1 << b) < d_in) ++b;
+  if (b == 0) return 0;
+  const unsigned long long mask = (b >= 64) ? ~0ull : (((unsigned long long)1 << b) - 1);
+  const int s = b / 2 > 1 ? b / 2 : 1;
+  unsigned long long key[3];
+  bcd_round_keys(seed, j, t, key);
+  unsigned long long v = (unsigned long long)x;
+  do {
+    for (int r = 0; r < 3; ++r) {
+      v = (v * (2ull * key[r] + 1ull) + (key[r] >> 33)) & mask;
+      v ^= v >> s;
+    }
+  } while (v >= (unsigned long long)d_in);
+  return (i64)v;
+}
+
+/* Q in/out.  k: block size (d_in % k == 0, k <= 4).  steps_per_col: T.      */
+/* moves_per_col, loss_before, loss_after: [d_out] (may be NULL); the losses */
+/* are recomputed from scratch as e^T H e.                                   */
+int cdqo_bcd_solve(const float* H, const double* W, i64 d_in, i64 d_out, int bits, i64 group_size,
+                   const float* scale, const float* zero, uint8_t* Q, int k, i64 steps_per_col,
+                   unsigned long long seed, i64* moves_per_col, double* loss_before, double* loss_after) {
+  if (!H || !W || !scale || !zero || !Q || bits < 1 || bits > 8 || k < 1 || k > 4) return 1;
+  const i64 g = group_size > 0 ? group_size : d_in;
+  if (d_in % g || d_in % k) return 2;
+  const i64 ng = d_in / g, nb = d_in / k;
+  const int L = (1 << bits) - 1;
+  i64 ncomb = 1;
+  for (int c = 0; c < k; ++c) ncomb *= (L + 1);
+#pragma omp parallel
+  {
+    double* w = (double*)malloc(sizeof(double) * d_in);
+    double* e = (double*)malloc(sizeof(double) * d_in);
+    double* G = (double*)malloc(sizeof(double) * d_in);
+    double* he = (double*)malloc(sizeof(double) * d_in);
+    uint8_t* q = (uint8_t*)malloc(d_in);
+    float* a = (float*)malloc(sizeof(float) * ng);
+    float* b = (float*)malloc(sizeof(float) * ng);
+#pragma omp for schedule(dynamic, 1)
+    for (i64 j = 0; j < d_out; ++j) {
+      for (i64 i = 0; i < d_in; ++i) { w[i] = W[i * d_out + j]; q[i] = Q[i * d_out + j]; }
+      for (i64 t = 0; t < ng; ++t) { a[t] = scale[t * d_out + j]; b[t] = zero[t * d_out + j]; }
+      residual(w, q, a, b, d_in, g, e);
+      const double l0 = quad_form(H, e, d_in, he);
+      if (loss_before) loss_before[j] = l0;
+      for (i64 p = 0; p < d_in; ++p) G[p] = 2.0 * he[p];
+      i64 moves = 0;
+      for (i64 t = 0; t < steps_per_col; ++t) {
+        double best = 0.0;
+        i64 best_min = -1;
+        i64 bm[4] = {0, 0, 0, 0};
+        int br[4] = {0, 0, 0, 0};
+        for (i64 u = 0; u < nb; ++u) {
+          i64 m[4];
+          for (int c = 0; c < k; ++c) m[c] = cdqo_bcd_perm(u * k + c, d_in, seed, j, t);
+          for (int c = 1; c < k; ++c) /* ascending coordinates */
+            for (int z = c; z > 0 && m[z] < m[z - 1]; --z) { const i64 tmp = m[z]; m[z] = m[z - 1]; m[z - 1] = tmp; }
+          for (i64 comb = 0; comb < ncomb; ++comb) {
+            int r[4];
+            i64 rest = comb;
+            for (int c = k - 1; c >= 0; --c) { r[c] = (int)(rest % (L + 1)); rest /= (L + 1); } /* first coordinate most significant */
+            double d[4];
+            int same = 1;
+            for (int c = 0; c < k; ++c) {
+              d[c] = (double)a[m[c] / g] * (double)(r[c] - (int)q[m[c]]);
+              if (r[c] != (int)q[m[c]]) same = 0;
+            }
+            if (same) continue;
+            double quad = 0.0, lin = 0.0;
+            for (int c = 0; c < k; ++c) {
+              for (int z = 0; z < k; ++z) quad = quad + (d[c] * d[z]) * (double)H[m[c] * d_in + m[z]];
+              lin = lin + d[c] * G[m[c]];
+            }
+            const double change = quad + lin;
+            if (change < best || (change == best && best_min >= 0 && m[0] < best_min && change < 0.0)) {
+              best = change; best_min = m[0];
+              for (int c = 0; c < k; ++c) { bm[c] = m[c]; br[c] = r[c]; }
+            }
+          }
+        }
+        if (best_min < 0) continue; /* this partition has no improving block */
+        for (int c = 0; c < k; ++c) {
+          const double dc = (double)a[bm[c] / g] * (double)(br[c] - (int)q[bm[c]]);
+          q[bm[c]] = (uint8_t)br[c];
+          if (dc == 0.0) continue;
+          const float* row = H + bm[c] * d_in;
+          const double two_d = 2.0 * dc;
+          for (i64 p = 0; p < d_in; ++p) G[p] = G[p] + two_d * (double)row[p];
+        }
+        ++moves;
+      }
+      if (moves_per_col) moves_per_col[j] = moves;
+      for (i64 i = 0; i < d_in; ++i) Q[i * d_out + j] = q[i];
+      residual(w, q, a, b, d_in, g, e);
+      if (loss_after) loss_after[j] = quad_form(H, e, d_in, he);
+    }
+    free(w); free(e); free(G); free(he); free(q); free(a); free(b);
   }
   return 0;
 }

@@ -428,3 +428,74 @@ def test_owc_cd_against_brute_force_over_all_assignments():
             assert r1["moves"][j] == 1 and int(r1["gamma_idx"][bt, j]) == bk
         else:
             assert r1["moves"][j] == 0
+
+
+# ---------------------------------------------------------------- BCD with random blocks (Algorithm 2 / 5)
+def test_bcd_partition_is_a_permutation_and_varies():
+    for d in (1, 2, 7, 10, 64, 100, 257):
+        p0 = oracle.bcd_perm(d, 11, 3, 0)
+        assert sorted(p0.tolist()) == list(range(d))
+        if d >= 10:
+            assert not np.array_equal(p0, oracle.bcd_perm(d, 11, 3, 1))      # another step
+            assert not np.array_equal(p0, oracle.bcd_perm(d, 11, 4, 0))      # another column
+            assert not np.array_equal(p0, oracle.bcd_perm(d, 12, 3, 0))      # another seed
+    # every pair of coordinates gets paired at some step: the family is not stuck on a few partitions
+    d, seen = 12, set()
+    for t in range(400):
+        p = oracle.bcd_perm(d, 5, 0, t)
+        seen |= {tuple(sorted((int(p[2 * u]), int(p[2 * u + 1])))) for u in range(d // 2)}
+    assert len(seen) == d * (d - 1) // 2
+
+
+@pytest.mark.parametrize("bits,g", [(2, 0), (3, 8), (4, 0)])
+def test_bcd_with_block_size_one_is_the_greedy_descent(bits, g):
+    X, W, H32, init = _setup(70, 120, 24, 7, bits, g)
+    cd = oracle.cd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], 30, g)
+    b1 = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], 1, 30, seed=9, group_size=g)
+    assert np.array_equal(b1["Q"], cd["Q"]) and b1["moves"].sum() == cd["committed"]
+
+
+@pytest.mark.parametrize("bits,g,k", [(2, 0, 2), (3, 6, 2), (2, 0, 3)])
+def test_bcd_step_is_the_best_block_move_and_loss_is_the_loss_from_x(bits, g, k):
+    d_in, d_out = 12, 5
+    X, W, H32, init = _setup(71, 90, d_in, d_out, bits, g)
+    a = _expand(init["scale"], d_in); b = _expand(init["zero"], d_in)
+    Hd = H32.astype(np.float64); Wd = W.astype(np.float64)
+    seed = 21
+    one = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], k, 1, seed=seed, group_size=g)
+    np.testing.assert_allclose(one["loss_after"], _direct_loss(X, W, init["scale"], init["zero"], one["Q"]), rtol=1e-5)
+    for j in range(d_out):
+        # brute force over the blocks of pi(., step 0) and all level assignments, loss from the definition
+        q0 = init["Q"][:, j].astype(np.int64)
+        base = (a[:, j] * q0 + b[:, j] - Wd[:, j]); base = base @ Hd @ base
+        perm = oracle.bcd_perm(d_in, seed, j, 0)
+        best, bq = base, q0
+        for u in range(d_in // k):
+            blk = sorted(int(x) for x in perm[k * u:k * u + k])
+            for r in itertools.product(range(2 ** bits), repeat=k):
+                q = q0.copy(); q[blk] = r
+                e = a[:, j] * q + b[:, j] - Wd[:, j]
+                l = e @ Hd @ e
+                if l < best * (1 - 1e-12):
+                    best, bq = l, q
+        np.testing.assert_allclose(one["loss_after"][j], best, rtol=1e-9)
+        assert one["moves"][j] == (0 if bq is q0 else 1)
+    # many steps: the loss never rises and the moves are counted
+    many = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], k, 40, seed=seed, group_size=g)
+    assert (many["loss_after"] <= one["loss_after"] * (1 + 1e-12)).all()
+    prev = init["Q"]
+    lprev = many["loss_before"]
+    for T in (5, 10, 20, 40):     # prefixes of the same run (the partition depends on the step index only)
+        r = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], k, T, seed=seed, group_size=g)
+        assert (r["loss_after"] <= lprev * (1 + 1e-12)).all()
+        lprev = r["loss_after"]
+    assert np.array_equal(r["Q"], many["Q"])
+
+
+def test_bcd_from_the_greedy_solution_never_worse():
+    X, W, H32, init = _setup(72, 200, 32, 10, 2)
+    cd = oracle.cd_solve(H32, W, 2, init["scale"], init["zero"], init["Q"], 64)
+    b2 = oracle.bcd_solve(H32, W, 2, init["scale"], init["zero"], cd["Q"], 2, 128, seed=1)
+    _, per = oracle.layer_loss(H32, W, init["scale"], init["zero"], cd["Q"])
+    np.testing.assert_allclose(b2["loss_before"], per, rtol=1e-12)
+    assert (b2["loss_after"] <= b2["loss_before"]).all() and b2["moves"].sum() > 0
