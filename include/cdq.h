@@ -189,6 +189,37 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
                               cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Block coordinate descent with random blocks (paper: Algorithm 2; Algorithm 5 for sub-channel
+ * grids), weight-unit form as above.  Step t of column j cuts the d_in coordinates into
+ * d_in / block blocks by a pseudo-random permutation pi (block u holds pi(block u), ...,
+ * pi(block u + block - 1)); every block b and every assignment r of levels to its coordinates is
+ * scored, with d = a (r - q) on b,
+ *     change = d^T H_bb d + d^T G_b,
+ * the most negative change is applied (ties: the block whose lowest coordinate is lowest, then
+ * the lowest levels in ascending order of the block's coordinates) and G += 2 sum_i d_i H[i,:].
+ * A step whose partition holds no improving block changes nothing; the descent runs all
+ * steps_per_col steps.
+ *   block  1: the greedy descent of cdq_cd_solve_steps (seed unused); 2: pairs.  Other sizes
+ *          return CDQ_ERR_UNSUPPORTED; d_in % block != 0 returns CDQ_ERR_SHAPE; pairs need
+ *          d_in <= 32768.
+ *   seed   pi is a counter-based bijection of {0..d_in-1}: with b = ceil(log2 d_in) bits, three
+ *          rounds  x <- (x (2 K_r + 1) + (K_r >> 33)) mod 2^b;  x <- x xor (x >> max(1, b / 2)),
+ *          repeated while x >= d_in, with K_r = splitmix64(base xor (4 t + r)) and
+ *          base = splitmix64(seed xor splitmix64(j)).  The same (seed, j, t) gives the same
+ *          partition on every run and on every implementation of this definition.
+ *   stats  as for cdq_cd_solve; columns_converged is 0 for block > 1 (no early stop).
+ * Workspace: that of CDQ_CALL_CD_SOLVE.
+ * FAST: fp32 scoring from an fp64 gradient, one pass over the levels of the block's lower
+ * coordinate with the other level in closed form; VERIFY: fp64 scan of all (L+1)^2 assignments
+ * in the fixed order, bit-reproducible.
+ */
+cdq_status cdq_bcd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                         long long ldw, const cdq_grid_desc* grid, const float* scale,
+                         const float* zero, unsigned char* Q, int block, long long steps_per_col,
+                         unsigned long long seed, cdq_mode mode, cdq_cd_stats* stats, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/*
  * Layer loss sum_j e_j^T H e_j with e = W_hat - W (paper: Eq. 1 written with
  * H = X^T X; the objective value the paper reports for a solution).
  *   loss     host pointer to one double, may be NULL.

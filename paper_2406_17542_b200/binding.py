@@ -24,7 +24,7 @@ MODE_FAST, MODE_FP64_VERIFY = 0, 1
 CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD = 0, 1, 2, 3, 4
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_layer_loss", "cdq_layer_loss_static",
+EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version"]
 
@@ -89,6 +89,9 @@ def load():
                                     ci, vp, sz, vp]
     lib.cdq_cd_solve.restype = ci
     lib.cdq_cd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
+    lib.cdq_bcd_solve.restype = ci
+    lib.cdq_bcd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ll, ctypes.c_ulonglong, ci,
+                                  ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_cd_solve_steps.restype = ci
     lib.cdq_cd_solve_steps.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_layer_loss.restype = ci
@@ -235,6 +238,30 @@ def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tens
             scale.data_ptr(), zero.data_ptr(), Q.data_ptr(), int(passes if steps_per_col is None else steps_per_col),
             _MODES[mode], ctypes.byref(stats) if want_stats else None, wptr, wbytes, _stream())
     _check(st, "cdq_cd_solve")
+    if not want_stats:
+        return None
+    return {"steps": stats.steps, "committed": stats.committed, "columns_converged": stats.columns_converged,
+            "loss_before": stats.loss_before, "loss_after": stats.loss_after, "kernel_ms": stats.kernel_ms}
+
+
+def cdq_bcd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,
+                  Q: torch.Tensor, block: int, steps_per_col: int, seed: int = 0, mode="fast",
+                  want_stats: bool = True, ws: Workspace | None = None):
+    """Block coordinate descent with random blocks of `block` coordinates; Q is updated in place."""
+    _need_cuda(H, W, scale, zero, Q)
+    d_in, d_out = W.shape
+    assert H.shape == (d_in, d_in) and H.is_contiguous() and H.dtype == torch.float32
+    assert Q.shape == (d_in, d_out) and Q.is_contiguous() and Q.dtype == torch.uint8
+    assert scale.is_contiguous() and zero.is_contiguous() and W.stride(1) == 1
+    gd = grid.c()
+    stats = cdq_cd_stats()
+    ws = ws or _default_ws
+    wptr, wbytes = ws.get(workspace_bytes(CALL_CD_SOLVE, 0, d_in, d_out, grid, mode), W.device)
+    st = load().cdq_bcd_solve(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), ctypes.byref(gd),
+                              scale.data_ptr(), zero.data_ptr(), Q.data_ptr(), int(block), int(steps_per_col),
+                              int(seed) & 0xFFFFFFFFFFFFFFFF, _MODES[mode], ctypes.byref(stats) if want_stats else None,
+                              wptr, wbytes, _stream())
+    _check(st, "cdq_bcd_solve")
     if not want_stats:
         return None
     return {"steps": stats.steps, "committed": stats.committed, "columns_converged": stats.columns_converged,

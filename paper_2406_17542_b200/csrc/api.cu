@@ -271,10 +271,13 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
 
 static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
                                 const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
-                                long long steps_per_col, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes,
-                                void* stream) {
+                                long long steps_per_col, int block, unsigned long long seed, cdq_mode mode,
+                                cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
   if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || steps_per_col < 0)
     return CDQ_ERR_INVALID_ARG;
+  if (block < 1) return CDQ_ERR_INVALID_ARG;
+  if (block > 1 && d_in % block) return CDQ_ERR_SHAPE;
+  if (block > 1 && !bcd_supported(d_in, block)) return CDQ_ERR_UNSUPPORTED;
   cdq_status s = check_layer_shape(d_in, d_out, ldw);
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);
@@ -317,7 +320,12 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   // shapes the fast kernels do not cover (a group size that is not a multiple of 4, very long
   // columns) take the fixed-order fp64 kernel: slower, same result
   const bool fast_cd = mode == CDQ_MODE_FAST && cd_fast_supported(d_in, ly.g);
-  if (fast_cd) {
+  if (block > 1) {
+    const bool fast = mode == CDQ_MODE_FAST;
+    if (fast) CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
+    if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
+    CDQ_CUDA(launch_bcd(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, seed, fast, ctr, st));
+  } else if (fast_cd) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
     CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, ctr, st));
@@ -352,16 +360,24 @@ cdq_status cdq_cd_solve(const float* H, const void* W, cdq_dtype wt, long long d
                         const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
                         int passes, cdq_mode mode, cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
   if (passes < 0) return CDQ_ERR_INVALID_ARG;
-  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, (long long)passes * d_in, mode, stats, ws,
-                       ws_bytes, stream);
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, (long long)passes * d_in, 1, 0ull, mode, stats,
+                       ws, ws_bytes, stream);
 }
 
 cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
                               long long ldw, const cdq_grid_desc* grid, const float* scale, const float* zero,
                               unsigned char* Q, long long steps_per_col, cdq_mode mode, cdq_cd_stats* stats, void* ws,
                               size_t ws_bytes, void* stream) {
-  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, mode, stats, ws, ws_bytes,
-                       stream);
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, 1, 0ull, mode, stats, ws,
+                       ws_bytes, stream);
+}
+
+cdq_status cdq_bcd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
+                         const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q, int block,
+                         long long steps_per_col, unsigned long long seed, cdq_mode mode, cdq_cd_stats* stats, void* ws,
+                         size_t ws_bytes, void* stream) {
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, block, seed, mode, stats, ws,
+                       ws_bytes, stream);
 }
 
 cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,

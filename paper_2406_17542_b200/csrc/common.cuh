@@ -123,6 +123,11 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
                            CdCounters* ctr, cudaStream_t st);
 cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                              long long steps_per_col, CdCounters* ctr, cudaStream_t st);
+// bcd_kernel.cu: random blocks of two coordinates (Algorithm 2 / 5)
+bool bcd_supported(long long d_in, int block);
+cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq, const float* hdiag,
+                       const float* hs, long long steps_per_col, unsigned long long seed, bool fast, CdCounters* ctr,
+                       cudaStream_t st);
 cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st);  // ascending order
 cudaError_t launch_sum_f64_tree(const double* v, long long n, double* out, cudaStream_t st);  // fixed tree order
 

@@ -1,0 +1,146 @@
+"""GPU parity of the block coordinate descent with random pairs (paper: Algorithm 2 / Algorithm 5)
+against the fp64 CPU oracle on the same seeded layers, the same starting codes and the same
+(seed, column, step) partitions.
+
+Bars as for the greedy descent: the fp64 verification mode bit-exact; the production mode at
+least 99.9 % equal codes and the layer loss within 1e-4 relative."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2406_17542_b200 import binding as B
+from paper_2406_17542_b200 import inputs
+from tests.util import grid_of
+
+pytestmark = pytest.mark.gpu
+
+CODE_AGREE = 0.999
+LOSS_RTOL = 1e-4
+
+
+def _layer(d_in, d_out, n, bits, g, seed):
+    cfg = inputs.CONFIGS["C0"].scaled(d_in=d_in, d_out=d_out, n=n, bits=bits, group_size=g, passes=1, seed=seed,
+                                      n_clip=1, clip_lo=1.0, clip_hi=1.0)
+    X, W = inputs.make_layer(cfg)
+    _, H32 = oracle.hessian(X, 0.0)
+    init = oracle.init_rtn(W, bits, g, 1, 1.0, 1.0)
+    return cfg, W, H32, init
+
+
+def _gpu_bcd(cfg, W, H32, init, block, steps, seed, mode):
+    dev = "cuda:0"
+    Hd = torch.from_numpy(np.ascontiguousarray(H32)).to(dev)
+    Wd = W.to(dev)
+    scale = torch.from_numpy(init["scale"]).to(dev)
+    zero = torch.from_numpy(init["zero"]).to(dev)
+    Q = torch.from_numpy(init["Q"]).to(dev).clone()
+    g = grid_of(cfg)
+    stats = B.cdq_bcd_solve(Hd, Wd, g, scale, zero, Q, block, steps, seed=seed, mode=mode)
+    loss = B.cdq_layer_loss(Hd, Wd, g, scale, zero, Q, mode=mode)
+    assert B.load().cdq_last_device_status() == 0
+    return Q.cpu().numpy(), stats, loss
+
+
+@pytest.mark.parametrize("d_in,d_out,n,bits,g,steps", [
+    (2, 5, 8, 2, 0, 3), (6, 4, 40, 3, 0, 12), (34, 17, 200, 3, 17, 40), (64, 24, 300, 4, 0, 96),
+    (96, 130, 500, 2, 32, 150), (520, 40, 1200, 2, 0, 300), (1024, 20, 2500, 3, 128, 200),
+])
+def test_pairs_verify_mode_is_bit_exact(d_in, d_out, n, bits, g, steps):
+    cfg, W, H32, init = _layer(d_in, d_out, n, bits, g, seed=300 + d_in)
+    ref = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], 2, steps, seed=77, group_size=g)
+    Q, stats, loss = _gpu_bcd(cfg, W, H32, init, 2, steps, 77, "verify")
+    assert np.array_equal(Q, ref["Q"])
+    assert stats["committed"] == int(ref["moves"].sum())
+    assert stats["steps"] == steps * d_out
+    np.testing.assert_allclose(stats["loss_before"], ref["loss_before"].sum(), rtol=1e-12)
+    np.testing.assert_allclose(stats["loss_after"], ref["loss_after"].sum(), rtol=1e-9)
+    np.testing.assert_allclose(loss, ref["loss_after"].sum(), rtol=1e-12)
+
+
+@pytest.mark.parametrize("d_in,d_out,n,bits,g,steps", [
+    (256, 64, 800, 2, 0, 256), (640, 96, 1600, 3, 128, 400), (1024, 48, 2500, 4, 0, 512),
+    (2048, 40, 4500, 2, 128, 600), (4608, 12, 6000, 3, 0, 300),
+])
+def test_pairs_fast_mode(d_in, d_out, n, bits, g, steps):
+    cfg, W, H32, init = _layer(d_in, d_out, n, bits, g, seed=400 + d_in)
+    ref = oracle.bcd_solve(H32, W, bits, init["scale"], init["zero"], init["Q"], 2, steps, seed=5, group_size=g)
+    Q, stats, loss = _gpu_bcd(cfg, W, H32, init, 2, steps, 5, "fast")
+    agree = float((Q == ref["Q"]).mean())
+    assert agree >= CODE_AGREE, agree
+    ref_loss = ref["loss_after"].sum()
+    assert abs(loss - ref_loss) <= LOSS_RTOL * ref_loss
+    assert stats["loss_after"] <= stats["loss_before"]
+    np.testing.assert_allclose(stats["loss_after"], loss, rtol=1e-5)
+    assert abs(stats["committed"] - int(ref["moves"].sum())) <= 0.01 * ref["moves"].sum() + 2
+
+
+def test_block_of_one_is_the_greedy_descent_and_seeds_matter():
+    cfg, W, H32, init = _layer(512, 64, 1500, 3, 128, seed=41)
+    dev = "cuda:0"
+    Hd = torch.from_numpy(np.ascontiguousarray(H32)).to(dev)
+    Wd, g = W.to(dev), grid_of(cfg)
+    scale, zero = torch.from_numpy(init["scale"]).to(dev), torch.from_numpy(init["zero"]).to(dev)
+    Qa = torch.from_numpy(init["Q"]).to(dev).clone()
+    Qb = Qa.clone()
+    B.cdq_cd_solve(Hd, Wd, g, scale, zero, Qa, 0, steps_per_col=200)
+    B.cdq_bcd_solve(Hd, Wd, g, scale, zero, Qb, 1, 200, seed=9)
+    assert torch.equal(Qa, Qb)
+    Q1, _, l1 = _gpu_bcd(cfg, W, H32, init, 2, 200, 1, "fast")
+    Q2, _, l2 = _gpu_bcd(cfg, W, H32, init, 2, 200, 2, "fast")
+    Q1b, _, l1b = _gpu_bcd(cfg, W, H32, init, 2, 200, 1, "fast")
+    assert np.array_equal(Q1, Q1b) and l1 == l1b     # same seed: same run
+    assert not np.array_equal(Q1, Q2)                # another seed: other partitions
+
+
+def test_pairs_after_the_greedy_descent_do_not_raise_the_loss():
+    cfg, W, H32, init = _layer(768, 80, 2000, 2, 0, seed=43)
+    dev = "cuda:0"
+    Hd = torch.from_numpy(np.ascontiguousarray(H32)).to(dev)
+    Wd, g = W.to(dev), grid_of(cfg)
+    scale, zero = torch.from_numpy(init["scale"]).to(dev), torch.from_numpy(init["zero"]).to(dev)
+    Q = torch.from_numpy(init["Q"]).to(dev).clone()
+    B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, 2)
+    l_cd = B.cdq_layer_loss(Hd, Wd, g, scale, zero, Q)
+    stats = B.cdq_bcd_solve(Hd, Wd, g, scale, zero, Q, 2, 768, seed=3)
+    l_bcd = B.cdq_layer_loss(Hd, Wd, g, scale, zero, Q)
+    assert l_bcd <= l_cd * (1 + 1e-9)
+    assert stats["committed"] > 0 and l_bcd < l_cd   # pairs leave minima that single moves cannot
+    assert int(Q.max()) <= 3
+
+
+def test_bad_block_arguments_are_refused():
+    cfg, W, H32, init = _layer(33, 4, 100, 3, 0, seed=47)
+    dev = "cuda:0"
+    Hd = torch.from_numpy(np.ascontiguousarray(H32)).to(dev)
+    Wd, g = W.to(dev), grid_of(cfg)
+    scale, zero = torch.from_numpy(init["scale"]).to(dev), torch.from_numpy(init["zero"]).to(dev)
+    Q = torch.from_numpy(init["Q"]).to(dev).clone()
+    for block in (0, 2, 3):     # 0: invalid; 2: 33 is odd; 3: not built
+        with pytest.raises(RuntimeError):
+            B.cdq_bcd_solve(Hd, Wd, g, scale, zero, Q, block, 10)
+    assert np.array_equal(Q.cpu().numpy(), init["Q"])
+
+
+def test_gradient_in_global_memory_gives_the_same_codes():
+    """The path of layers whose column does not fit in shared memory, forced on a small layer
+    in a child process (the switch is read once per process)."""
+    code = (
+        "import numpy as np, torch, oracle\n"
+        "from tests.test_bcd_gpu import _layer, _gpu_bcd\n"
+        "cfg, W, H32, init = _layer(640, 40, 1600, 3, 128, seed=53)\n"
+        "ref = oracle.bcd_solve(H32, W, 3, init['scale'], init['zero'], init['Q'], 2, 300, seed=11, group_size=128)\n"
+        "Q, stats, loss = _gpu_bcd(cfg, W, H32, init, 2, 300, 11, 'fast')\n"
+        "agree = float((Q == ref['Q']).mean())\n"
+        "assert agree >= 0.999, agree\n"
+        "assert abs(loss - ref['loss_after'].sum()) <= 1e-4 * ref['loss_after'].sum()\n"
+        "print('ok', agree)\n"
+    )
+    env = dict(os.environ, CDQ_BCD_G="global")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout + r.stderr
