@@ -163,6 +163,9 @@ def main():
     ap.add_argument("--budget-div", type=int, default=0,
                     help="descent budget T = d_in / DIV steps per column (the paper's fewer-iterations study) "
                          "instead of the config's passes * d_in")
+    ap.add_argument("--block", type=int, default=1, choices=[1, 2],
+                    help="1: greedy descent (the headline path); 2: BCD with random pairs (Algorithm 2 / 5) on the same "
+                         "budget of steps per column; no CPU baseline is timed for it")
     ap.add_argument("--init", default="rtn", choices=["rtn", "owc_cd"],
                     help="grid stage: cdq_init_rtn (MinMax / OWC as the config says) or cdq_init_owc_cd (Algorithm 3; "
                          "configs with a clipping grid)")
@@ -181,7 +184,8 @@ def main():
     workload = (f"{cfg.name}: d_in={cfg.d_in} d_out={cfg.d_out} n={cfg.n} X={cfg.x_dtype} W={cfg.w_dtype} "
                 f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}"
                 + (" init=OWC-CD" if args.init == "owc_cd" else "")
-                + (f" budget=d_in/{args.budget_div}" if args.budget_div > 0 else ""))
+                + (f" budget=d_in/{args.budget_div}" if args.budget_div > 0 else "")
+                + (" descent=BCD(k=2)" if args.block == 2 else ""))
 
     if args.impl == "reference":
         if rank != 0:
@@ -223,8 +227,11 @@ def main():
         else:
             scale, zero, Q, _ = B.cdq_init_rtn(Wd, grid, H=H if cfg.n_clip > 1 else None, ws=ws)
         ev[3].record()
-        stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
-                               steps_per_col=cfg.d_in // args.budget_div if args.budget_div > 0 else None)
+        budget = cfg.d_in // args.budget_div if args.budget_div > 0 else None
+        if args.block == 2:
+            stats = B.cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, budget or cfg.passes * cfg.d_in, seed=cfg.seed, ws=ws)
+        else:
+            stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws, steps_per_col=budget)
         ev[4].record()
         loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws)
         if host:
@@ -277,6 +284,8 @@ def main():
     mean = lambda v: sum(v) / len(v)
     cd_ms = mean(times["cd_kernel"])
     alg_bytes = algorithmic_bytes_cd(cfg, committed)
+    if args.block == 2:  # two rows per move at most, and one H_im per pair and step
+        alg_bytes += committed * 4.0 * cfg.d_in + stats["steps"] * 2.0 * cfg.d_in
     achieved = alg_bytes / (cd_ms * 1e-3) / 1e9
     h_in_l2 = 4.0 * cfg.d_in * cfg.d_in < 100e6
     hess_ms = mean(times["hessian"])
@@ -305,10 +314,10 @@ def main():
                     "executed_frac_of_bf16_sustained_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                     "executed_frac_of_bf16_burst_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                     "note": "symmetric rank-k update: only lower-triangle tiles are computed; the fraction counts executed flops only"},
-        "roofline": {"kernel": "cd_fast_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        "roofline": {"kernel": "bcd2_kernel" if args.block == 2 else "cd_fast_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes": alg_bytes,
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.block == 1 else None, "algorithmic_bytes": alg_bytes,
                      "note": ("H fits in L2 for this workload: rows are L2-served, the figure is effective GB/s"
                               if h_in_l2 else "H exceeds L2: rows stream from HBM")},
         "e2e": {"value": committed_all / (total_ms_e2e / args.steps * 1e-3), "unit": UNIT,
@@ -316,7 +325,7 @@ def main():
         "gpu_launches": kernel_launches(cfg) * args.steps,
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and args.block == 1:
         # about 5-10 s of Hessian and 5-10 s of descent on 8 host cores
         n_rows = min(cfg.n, max(1024, int(4.0e10 / (cfg.d_in * cfg.d_in))))
         n_cols = min(cfg.d_out, max(8, int(3.0e10 / (0.8 * cfg.d_in * cfg.d_in * (2 ** cfg.bits)))))

@@ -67,7 +67,8 @@ typedef enum {
   CDQ_CALL_INIT_RTN = 1,
   CDQ_CALL_CD_SOLVE = 2,
   CDQ_CALL_LAYER_LOSS = 3,
-  CDQ_CALL_INIT_OWC_CD = 4
+  CDQ_CALL_INIT_OWC_CD = 4,
+  CDQ_CALL_BCD_SOLVE = 5   /* n: steps per column */
 } cdq_call;
 
 /* Quantization grid (paper: c in "Notation"; group size g in the sub-channel
@@ -190,9 +191,9 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
 
 /*
  * Block coordinate descent with random blocks (paper: Algorithm 2; Algorithm 5 for sub-channel
- * grids), weight-unit form as above.  Step t of column j cuts the d_in coordinates into
- * d_in / block blocks by a pseudo-random permutation pi (block u holds pi(block u), ...,
- * pi(block u + block - 1)); every block b and every assignment r of levels to its coordinates is
+ * grids), weight-unit form as above.  Step t cuts the d_in coordinates into d_in / block blocks
+ * by a pseudo-random permutation pi (block u holds pi(block u), ..., pi(block u + block - 1)),
+ * drawn once per step for all columns; every block b and every assignment r of levels to its coordinates is
  * scored, with d = a (r - q) on b,
  *     change = d^T H_bb d + d^T G_b,
  * the most negative change is applied (ties: the block whose lowest coordinate is lowest, then
@@ -204,11 +205,13 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
  *          d_in <= 32768.
  *   seed   pi is a counter-based bijection of {0..d_in-1}: with b = ceil(log2 d_in) bits, three
  *          rounds  x <- (x (2 K_r + 1) + (K_r >> 33)) mod 2^b;  x <- x xor (x >> max(1, b / 2)),
- *          repeated while x >= d_in, with K_r = splitmix64(base xor (4 t + r)) and
- *          base = splitmix64(seed xor splitmix64(j)).  The same (seed, j, t) gives the same
- *          partition on every run and on every implementation of this definition.
+ *          repeated while x >= d_in, with K_r = splitmix64(splitmix64(seed) xor (4 t + r)).
+ *          The same (seed, t) gives the same partition on every run and on every
+ *          implementation of this definition.
  *   stats  as for cdq_cd_solve; columns_converged is 0 for block > 1 (no early stop).
- * Workspace: that of CDQ_CALL_CD_SOLVE.
+ * Workspace: cdq_workspace_bytes(CDQ_CALL_BCD_SOLVE, steps_per_col, ...); with block == 2 the
+ * production mode lists the pairs of all steps there (8 d_in bytes per step), so
+ * steps_per_col <= 65535.
  * FAST: fp32 scoring from an fp64 gradient, one pass over the levels of the block's lower
  * coordinate with the other level in closed form; VERIFY: fp64 scan of all (L+1)^2 assignments
  * in the fixed order, bit-reproducible.

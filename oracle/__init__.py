@@ -59,7 +59,7 @@ def _load():
     lib.cdqo_hessian.argtypes = [_dp, _i64, _i64, ctypes.c_double, _dp, _fp]
     lib.cdqo_hessian_entries.argtypes = [_dp, _i64, _i64, _i64p, _i64p, _i64, _dp]
     lib.cdqo_bcd_perm.restype = _i64
-    lib.cdqo_bcd_perm.argtypes = [_i64, _i64, ctypes.c_ulonglong, _i64, _i64]
+    lib.cdqo_bcd_perm.argtypes = [_i64, _i64, ctypes.c_ulonglong, _i64]
     lib.cdqo_bcd_solve.argtypes = [_fp, _dp, _i64, _i64, ctypes.c_int, _i64, _fp, _fp, _u8p, ctypes.c_int, _i64,
                                    ctypes.c_ulonglong, _i64p, _dp, _dp]
     lib.cdqo_owc_cd.argtypes = [_dp, _i64, _i64, _fp, ctypes.c_int, _i64, ctypes.c_int, ctypes.c_double,
@@ -182,10 +182,10 @@ def owc_cd(H, W, bits: int, group_size: int, n_clip: int, clip_lo: float, clip_h
             "loss_before": lb, "loss_after": la}
 
 
-def bcd_perm(d_in: int, seed: int, col: int, step: int) -> np.ndarray:
-    """The pseudo-random permutation pi that cuts the coordinates into blocks at one step of one column."""
+def bcd_perm(d_in: int, seed: int, step: int) -> np.ndarray:
+    """The pseudo-random permutation pi that cuts the coordinates into blocks at one step (the same for every column)."""
     lib = _load()
-    return np.array([lib.cdqo_bcd_perm(x, d_in, seed, col, step) for x in range(d_in)], dtype=np.int64)
+    return np.array([lib.cdqo_bcd_perm(x, d_in, seed, step) for x in range(d_in)], dtype=np.int64)
 
 
 def bcd_solve(H, W, bits: int, scale, zero, Q, k: int, steps_per_col: int, seed: int = 0, group_size: int = 0) -> dict:

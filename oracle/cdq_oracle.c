@@ -55,7 +55,7 @@
  * tracked loss against the loss recomputed from X; one group == the OWC grid
  * search; brute force over all assignments of grid points to groups; first
  * change == best single-group change; convergence == no improving change.
- * BCD: the partition is a permutation that varies with step, column and seed
+ * BCD: the partition is a permutation that varies with step and seed
  * and reaches every pair; block size 1 == the greedy descent; one step == the
  * brute-force best block move with the loss from the definition; prefixes of
  * a run are monotone.
@@ -583,8 +583,9 @@ int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
 /* BCD with random blocks (Algorithm 2; Algorithm 5 for sub-channel grids),  */
 /* block size k, weight-unit form as for the greedy descent above.           */
 /*                                                                           */
-/* Step t of column j: the coordinates are cut into d_in / k blocks by a     */
-/* pseudo-random permutation pi (block u = {pi(k u), ..., pi(k u + k - 1)}); */
+/* Step t: the coordinates are cut into d_in / k blocks by a pseudo-random   */
+/* permutation pi (block u = {pi(k u), ..., pi(k u + k - 1)}), drawn once    */
+/* per step for the whole layer (all columns see the same partition);        */
 /* for every block and every assignment r of levels to its coordinates, with */
 /* d_i = a_i (r_i - q_i),                                                    */
 /*     change = sum_i d_i^2 H_ii + 2 sum_{i<m} d_i d_m H_im + sum_i d_i G_i  */
@@ -597,12 +598,14 @@ int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
 /*    implementation: with b = bits of d_in - 1 and mask = 2^b - 1, three    */
 /*    rounds  x <- (x * (2 K_r + 1) + (K_r >> 33)) & mask;  x <- x ^ (x >> s) */
 /*    with                                                                   */
-/*    s = max(1, b / 2) and K_r = splitmix64(seed, j, t, r) (each round is a */
+/*    s = max(1, b / 2) and K_r = splitmix64(seed, t, r) (each round is a    */
 /*    bijection of b-bit words), repeated while x >= d_in (cycle walking).   */
+/*    The column is not part of the key: the algorithm is stated for one     */
+/*    vector and applied to a layer as a batch, one draw per step;           */
 /*    splitmix64 is the published finaliser  z += 0x9E3779B97F4A7C15;        */
 /*    z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9; z = (z ^ z >> 27) *            */
 /*    0x94D049BB133111EB; z ^ z >> 31  applied to                            */
-/*    seed ^ (j << 40) ^ (t << 8) ^ r folded as below;                       */
+/*    splitmix64(seed) ^ (4 t + r);                                          */
 /*  - a step whose partition holds no improving block changes nothing and    */
 /*    the next step draws the next partition (the loop does not stop);       */
 /*  - ties: the block whose smallest coordinate is lowest, then the          */
@@ -616,20 +619,20 @@ static unsigned long long cdqo_splitmix64(unsigned long long z) {
   z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
   return z ^ (z >> 31);
 }
-/* keys of the three rounds for (seed, column, step) */
-static void bcd_round_keys(unsigned long long seed, i64 j, i64 t, unsigned long long key[3]) {
-  const unsigned long long base = cdqo_splitmix64(seed ^ cdqo_splitmix64((unsigned long long)j));
+/* keys of the three rounds for (seed, step) */
+static void bcd_round_keys(unsigned long long seed, i64 t, unsigned long long key[3]) {
+  const unsigned long long base = cdqo_splitmix64(seed);
   for (int r = 0; r < 3; ++r) key[r] = cdqo_splitmix64(base ^ (((unsigned long long)t << 2) | (unsigned long long)r));
 }
 /* pi(x) for the partition of step t; exported for the tests */
-i64 cdqo_bcd_perm(i64 x, i64 d_in, unsigned long long seed, i64 j, i64 t) {
+i64 cdqo_bcd_perm(i64 x, i64 d_in, unsigned long long seed, i64 t) {
   int b = 0;
   while (((i64)1 << b) < d_in) ++b;
   if (b == 0) return 0;
   const unsigned long long mask = (b >= 64) ? ~0ull : (((unsigned long long)1 << b) - 1);
   const int s = b / 2 > 1 ? b / 2 : 1;
   unsigned long long key[3];
-  bcd_round_keys(seed, j, t, key);
+  bcd_round_keys(seed, t, key);
   unsigned long long v = (unsigned long long)x;
   do {
     for (int r = 0; r < 3; ++r) {
@@ -678,7 +681,7 @@ int cdqo_bcd_solve(const float* H, const double* W, i64 d_in, i64 d_out, int bit
         int br[4] = {0, 0, 0, 0};
         for (i64 u = 0; u < nb; ++u) {
           i64 m[4];
-          for (int c = 0; c < k; ++c) m[c] = cdqo_bcd_perm(u * k + c, d_in, seed, j, t);
+          for (int c = 0; c < k; ++c) m[c] = cdqo_bcd_perm(u * k + c, d_in, seed, t);
           for (int c = 1; c < k; ++c) /* ascending coordinates */
             for (int z = c; z > 0 && m[z] < m[z - 1]; --z) { const i64 tmp = m[z]; m[z] = m[z - 1]; m[z - 1] = tmp; }
           for (i64 comb = 0; comb < ncomb; ++comb) {

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "CDQ_OK", 1: "CDQ_ERR_INVALID_ARG", 2: "CDQ_ERR_SHAPE", 3: "C
                 4: "CDQ_ERR_WORKSPACE", 5: "CDQ_ERR_CUDA", 6: "CDQ_ERR_TIMEOUT"}
 CDQ_F32, CDQ_BF16 = 0, 1
 MODE_FAST, MODE_FP64_VERIFY = 0, 1
-CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD = 0, 1, 2, 3, 4
+CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD, CALL_BCD_SOLVE = 0, 1, 2, 3, 4, 5
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
 EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
@@ -256,7 +256,7 @@ def cdq_bcd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Ten
     gd = grid.c()
     stats = cdq_cd_stats()
     ws = ws or _default_ws
-    wptr, wbytes = ws.get(workspace_bytes(CALL_CD_SOLVE, 0, d_in, d_out, grid, mode), W.device)
+    wptr, wbytes = ws.get(workspace_bytes(CALL_BCD_SOLVE, int(steps_per_col), d_in, d_out, grid, mode), W.device)
     st = load().cdq_bcd_solve(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), ctypes.byref(gd),
                               scale.data_ptr(), zero.data_ptr(), Q.data_ptr(), int(block), int(steps_per_col),
                               int(seed) & 0xFFFFFFFFFFFFFFFF, _MODES[mode], ctypes.byref(stats) if want_stats else None,

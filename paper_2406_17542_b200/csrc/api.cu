@@ -60,12 +60,12 @@ Layer make_layer(const float* H, const void* W, cdq_dtype wt, long long d_in, lo
 
 // Workspace of cdq_cd_solve / cdq_layer_loss.
 struct SolveWs {
-  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, hbuf, ebuf, total;
+  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, hbuf, ebuf, bcd_tab, total;
   long long ldg, d_pad;
   bool tc;        // H E on the int8 tensor cores
   int nh, ne, smax;
 };
-SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd) {
+SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd, long long bcd_steps = 0) {
   SolveWs w{};
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -90,6 +90,7 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
   w.col_loss = take(sizeof(double) * d_out);
   w.scalars = take(256);  // [0]: loss sum; [64..): CdCounters
+  if (bcd_steps > 0 && mode == CDQ_MODE_FAST) w.bcd_tab = take(bcd_table_bytes(d_in, bcd_steps));
   w.total = off;
   return w;
 }
@@ -198,6 +199,9 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
     case CDQ_CALL_CD_SOLVE:
       if (d_out < 1) return 0;
       return solve_ws_layout(d_in, d_out, mode, true).total;
+    case CDQ_CALL_BCD_SOLVE:  // n: steps per column
+      if (d_out < 1 || n < 0) return 0;
+      return solve_ws_layout(d_in, d_out, mode, true, n).total;
     case CDQ_CALL_LAYER_LOSS:
       if (d_out < 1) return 0;
       return solve_ws_layout(d_in, d_out, mode, false).total;
@@ -282,7 +286,8 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);
   if (s != CDQ_OK) return s;
-  const SolveWs L = solve_ws_layout(d_in, d_out, mode, true);
+  if (block > 1 && steps_per_col > 65535) return CDQ_ERR_UNSUPPORTED;
+  const SolveWs L = solve_ws_layout(d_in, d_out, mode, true, block > 1 ? steps_per_col : 0);
   s = check_ws(ws, ws_bytes, L.total);
   if (s != CDQ_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
@@ -324,7 +329,8 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
     const bool fast = mode == CDQ_MODE_FAST;
     if (fast) CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
-    CDQ_CUDA(launch_bcd(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, seed, fast, ctr, st));
+    CDQ_CUDA(launch_bcd(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, seed, fast, base + L.bcd_tab, ctr,
+                        st));
   } else if (fast_cd) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));

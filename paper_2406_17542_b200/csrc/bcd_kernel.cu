@@ -1,19 +1,23 @@
 // Block coordinate descent with random blocks of two coordinates, batched over all output
 // columns (paper: Algorithm 2; Algorithm 5 for sub-channel grids; weight-unit form).
 //
-// Step t of column j cuts the coordinates into d_in / 2 pairs by a counter-based bijection
-// of {0..d_in-1} keyed by (seed, j, t); every pair (i, m) is scored over all (L+1)^2
-// assignments of levels,
+// Step t cuts the coordinates into d_in / 2 pairs by a counter-based bijection of
+// {0..d_in-1} keyed by (seed, t), the same for every column; every pair (i, m) is scored over
+// all (L+1)^2 assignments of levels,
 //   change = d_i^2 H_ii + 2 d_i d_m H_im + d_m^2 H_mm + d_i g_i + d_m g_m,  d = a (r - q),
 // the most negative change of the step is applied and g += 2 d_i H[i, :] + 2 d_m H[m, :].
 //
 // One CTA owns one column at a time.  Pairs touch the gradient and the codes at random, so
 // both live in shared memory (gradient fp64, 8 bytes per coordinate; codes 1 byte); the rows
-// of H stream through registers, and the off-diagonal entry H_im of every pair of step t + 1
-// is gathered while step t is applied (the partition does not depend on the state).
-// The scan over the (L+1)^2 assignments takes one pass over the levels of the lower
-// coordinate; for each, the best level of the other is the clamped rounding of the vertex of
-// its parabola, as in the greedy descent.
+// of H stream through registers.  The partition does not depend on the state or the column,
+// so a kernel of its own lists, once per call, the pairs of every step with their
+// off-diagonal entry H_im (d_in / 2 scattered reads per step, which would otherwise be paid
+// per column and bound the descent by the rate of random DRAM reads) and with the two
+// diagonal entries; the descent reads that table in order (16 bytes per pair and pass).
+// The scan over the (L+1)^2 assignments fixes a level of the lower coordinate and takes the
+// best level of the other in closed form (the clamped rounding of the vertex of its parabola,
+// as in the greedy descent); convexity of the change in the pair bounds which levels of the
+// lower coordinate can still win, so only a few of them are visited.
 #include <cstdio>
 #include <cstdlib>
 
@@ -24,7 +28,7 @@ namespace cdq {
 
 // ---------------------------------------------------------------------------
 // The partition: x -> pi(x), three rounds of (odd multiply + add) mod 2^b and xor-shift on
-// b = ceil(log2 d_in) bits, keyed per (seed, column, step); values >= d_in walk the cycle
+// b = ceil(log2 d_in) bits, keyed per (seed, step); values >= d_in walk the cycle
 // until they fall below d_in (a bijection maps the cycle back to its start, so this ends).
 __host__ __device__ __forceinline__ unsigned long long splitmix64(unsigned long long z) {
   z += 0x9E3779B97F4A7C15ull;
@@ -85,14 +89,32 @@ __device__ __forceinline__ float2 ld_row2(const float* p) {
 }
 
 // ---------------------------------------------------------------------------
+// tab[t * nb + u] = (m0 | m1 << 16, bits of H[m0, m1], H[m0, m0], H[m1, m1]) with m0 < m1 the pair u
+// of step t (the diagonal with negative entries set to 0).
+__global__ void bcd2_table_kernel(const float* __restrict__ H, const float* __restrict__ hdiag, unsigned d_in,
+                                  unsigned long long seed, BcdShape shape, uint4* __restrict__ tab) {
+  const unsigned nb = d_in >> 1;
+  const unsigned u = blockIdx.x * blockDim.x + threadIdx.x;
+  const long long t = blockIdx.y;
+  if (u >= nb) return;
+  const BcdKeys keys = bcd_keys(splitmix64(seed), t);
+  unsigned m0 = bcd_perm(2 * u, d_in, shape.mask, shape.shift, keys);
+  unsigned m1 = bcd_perm(2 * u + 1, d_in, shape.mask, shape.shift, keys);
+  if (m1 < m0) { const unsigned x = m0; m0 = m1; m1 = x; }
+  tab[(size_t)t * nb + u] = make_uint4(m0 | (m1 << 16), __float_as_uint(ld_nc_f32(H + (size_t)m0 * d_in + m1)),
+                                       __float_as_uint(hdiag[m0]), __float_as_uint(hdiag[m1]));
+}
+
+// ---------------------------------------------------------------------------
 // PPT: pairs per thread (pair u = tid + NT * slot).  g_in_smem == 0: the gradient stays in
 // its global-memory column (layers whose column does not fit in shared memory).
 // a_in_smem == 0: the group scales are read from global memory.
 template <int PPT, int MAXNT, int MINB>
 __global__ void __launch_bounds__(MAXNT, MINB)
-bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, int a_in_smem) {
+bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_smem) {
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   __shared__ __align__(16) uint4 s_exch[2][32];
+  __shared__ unsigned s_bound[2][32];
   __shared__ int s_col;
 
   const int tid = threadIdx.x, NT = blockDim.x;
@@ -104,7 +126,7 @@ bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, 
   // shared memory: [gradient, 8 ldg bytes][codes, ldg bytes rounded to 16][scales, 4 ng bytes]
   double* g_smem = reinterpret_cast<double*>(dyn_smem);
   unsigned char* q_s = dyn_smem + (g_in_smem ? sizeof(double) * (size_t)p.ldg : 0);
-  float* a_smem = reinterpret_cast<float*>(q_s + ((p.ldg + 15) / 16) * 16);
+  float2* a_smem = reinterpret_cast<float2*>(q_s + ((p.ldg + 15) / 16) * 16);   // (a, 1 / a) per group
   auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
 
   unsigned long long my_moves = 0;
@@ -120,8 +142,6 @@ bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, 
 
     // ---- column state ----
     double* g_s = g_in_smem ? g_smem : p.G + j * p.ldg;
-    const float* a_ptr = a_in_smem ? a_smem : p.scale + j;
-    const long long a_stride = a_in_smem ? 1 : p.d_out;
     if (g_in_smem) {
       const double* gcol = p.G + j * p.ldg;
       for (unsigned i = tid; i < d_in; i += NT) g_s[i] = gcol[i];
@@ -131,64 +151,124 @@ bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, 
       for (unsigned i = tid; i < d_in; i += NT) q_s[i] = qcol[i];
     }
     if (a_in_smem)
-      for (int t = tid; t < (int)p.ng; t += NT) a_smem[t] = p.scale[(long long)t * p.d_out + j];
-    __syncthreads();
-    auto scale_of = [&](unsigned i) -> float { return a_ptr[(long long)group_of(i) * a_stride]; };
-
-    const unsigned long long base = splitmix64(seed ^ splitmix64((unsigned long long)j));
-    unsigned idx[PPT];   // m0 | m1 << 16, m0 < m1
-    float h01[PPT];
-    auto draw = [&](long long t) {
-      const BcdKeys keys = bcd_keys(base, t);
-#pragma unroll
-      for (int s = 0; s < PPT; ++s) {
-        const unsigned u = (unsigned)tid + (unsigned)NT * s;
-        idx[s] = 0; h01[s] = 0.f;
-        if (u < nb) {
-          unsigned m0 = bcd_perm(2 * u, d_in, shape.mask, shape.shift, keys);
-          unsigned m1 = bcd_perm(2 * u + 1, d_in, shape.mask, shape.shift, keys);
-          if (m1 < m0) { const unsigned x = m0; m0 = m1; m1 = x; }
-          idx[s] = m0 | (m1 << 16);
-          h01[s] = ld_nc_f32(p.H + (size_t)m0 * d_in + m1);
-        }
+      for (int t = tid; t < (int)p.ng; t += NT) {
+        const float a = p.scale[(long long)t * p.d_out + j];
+        a_smem[t] = make_float2(a, a > 0.f ? 1.0f / a : 0.f);
       }
+    __syncthreads();
+    auto scale_of = [&](unsigned i) -> float2 {
+      if (a_in_smem) return a_smem[group_of(i)];
+      const float a = p.scale[(long long)group_of(i) * p.d_out + j];
+      return make_float2(a, a > 0.f ? 1.0f / a : 0.f);
     };
 
     double col_dsum = 0.0;
     long long moves = 0;
     bool bad = false;
-    if (p.T > 0) draw(0);
     for (long long t = 0; t < p.T; ++t) {
-      // ---- best move of every pair of this thread ----
+      // ---- pass 1: the best move of each coordinate alone (the pair with the other level kept) ----
+      const uint4* trow = tab + (size_t)t * nb;
       float best = 0.f;
       unsigned bpk = kNoMove, bextra = 0;
 #pragma unroll
       for (int s = 0; s < PPT; ++s) {
         const unsigned u = (unsigned)tid + (unsigned)NT * s;
         if (u >= nb) continue;
-        const unsigned m0 = idx[s] & 0xFFFFu, m1 = idx[s] >> 16;
-        const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
-        const int q0 = q_s[m0], q1 = q_s[m1];
-        const float a0 = scale_of(m0), a1 = scale_of(m1);
-        const float H00 = __ldg(p.hdiag + m0), H11 = __ldg(p.hdiag + m1);
-        const float w1 = a1 > 0.f ? __ldg(p.hs + m1) / a1 : 0.f;   // 1 / (2 a H_mm)
-        const float h2 = 2.f * h01[s];
-        const float q1f = (float)q1;
-        float pbest = 0.f;
-        int pr0 = 0, pr1 = 0;
-        for (int r0 = 0; r0 <= p.L; ++r0) {
-          const float d0 = a0 * (float)(r0 - q0);
-          const float fixed = d0 * fmaf(d0, H00, g0);
-          const float g1p = fmaf(d0, h2, g1);            // gradient of the second coordinate once the first has moved
-          const float r1f = fminf(fmaxf(rintf(fmaf(-g1p, w1, q1f)), 0.f), Lf);
-          const float d1 = a1 * (r1f - q1f);
-          const float val = fmaf(d1, fmaf(d1, H11, g1p), fixed);
-          if (val < pbest) { pbest = val; pr0 = r0; pr1 = (int)r1f; }
+        const uint4 e = __ldg(trow + u);
+        const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
+        const unsigned q0 = q_s[m0], q1 = q_s[m1];
+        const unsigned extra_s = m1 | (q0 << 16) | (q1 << 24);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const unsigned mc = c ? m1 : m0;
+          const float gc = (float)g_s[mc], qf = (float)(c ? q1 : q0);
+          const float2 ac = scale_of(mc);
+          const float Hcc = __uint_as_float(c ? e.w : e.z);
+          const float hsc = Hcc > 0.f ? 0.5f / Hcc : 0.f;
+          const float rf = fminf(fmaxf(rintf(fmaf(-gc, hsc * ac.y, qf)), 0.f), Lf);
+          const float d = ac.x * (rf - qf);
+          const float val = d * fmaf(d, Hcc, gc);
+          const unsigned pk = (m0 << 16) | (c ? (q0 << 8) | (unsigned)rf : ((unsigned)rf << 8) | q1);
+          if (val < best || (val == best && val < 0.f && pk < bpk)) { best = val; bpk = pk; bextra = extra_s; }
         }
-        if (pbest < best || (pbest == best && pbest < 0.f && ((m0 << 16) < (bpk & 0xFFFF0000u)))) {
-          best = pbest;
-          bpk = (m0 << 16) | ((unsigned)pr0 << 8) | (unsigned)pr1;
-          bextra = m1 | ((unsigned)q0 << 16) | ((unsigned)q1 << 24);
+      }
+      // the best of them over the team bounds what a pair has to beat
+      float bound;
+      {
+        unsigned k1 = __reduce_min_sync(0xFFFFFFFFu, best < 0.f ? ~__float_as_uint(best) : kNoMove);
+        if (nwarps > 1) {
+          if (lane == 0) s_bound[xbuf][warp] = k1;
+          __syncthreads();
+          k1 = __reduce_min_sync(0xFFFFFFFFu, lane < nwarps ? s_bound[xbuf][lane] : kNoMove);
+        }
+        bound = k1 == kNoMove ? 0.f : __uint_as_float(~k1);
+      }
+
+      // ---- pass 2: pairs that can beat the bound ----
+#pragma unroll
+      for (int s = 0; s < PPT; ++s) {
+        const unsigned u = (unsigned)tid + (unsigned)NT * s;
+        if (u >= nb) continue;
+        const uint4 e = __ldg(trow + u);
+        const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
+        const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
+        const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
+        const float h2 = 2.f * h01;
+        // The change is convex in the pair (H is positive semi-definite): no assignment does
+        // better than the free minimum -N / (4 det), N = g0^2 H11 - 2 g0 g1 H01 + g1^2 H00.
+        // A pair whose 2 x 2 block of H is close to singular in fp32 is never skipped and is
+        // scanned in full.
+        const float det = fmaf(H00, H11, -h01 * h01);
+        const bool full = !(det > 1e-4f * H00 * H11);
+        const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -g0 * g1 * h2));
+        if (!full && 1.001f * N < -4.f * bound * det) continue;
+        const int q0 = q_s[m0], q1 = q_s[m1];
+        const float2 a0 = scale_of(m0), a1 = scale_of(m1);
+        const unsigned extra_s = m1 | ((unsigned)q0 << 16) | ((unsigned)q1 << 24);
+        // S: the coordinate whose levels are scanned (the one with the larger a^2 H_ii, so that
+        // few of its levels can win); F: the other, whose level follows in closed form
+        const bool swap = !full && a1.x * a1.x * H11 > a0.x * a0.x * H00;
+        const float gS = swap ? g1 : g0, gF = swap ? g0 : g1;
+        const int qS = swap ? q1 : q0, qF = swap ? q0 : q1;
+        const float aS = swap ? a1.x : a0.x, aF = swap ? a0.x : a1.x;
+        const float HSS = swap ? H11 : H00, HFF = swap ? H00 : H11;
+        const float wF = HFF > 0.f ? 0.5f / HFF * (swap ? a0.y : a1.y) : 0.f;   // 1 / (2 a H_ii)
+        const float qFf = (float)qF;
+        // phi(rS): the change with F free in [0, L] (not rounded): convex in rS and a lower
+        // bound of the rounded change, so the scan walks outwards from qS and stops on a side
+        // once phi has passed the bound and no longer falls.
+        auto eval = [&](int rS) -> float {
+          const float dS = aS * (float)(rS - qS);
+          const float fixed = dS * fmaf(dS, HSS, gS);
+          const float gFp = fmaf(dS, h2, gF);            // gradient of F once S has moved
+          const float x = fminf(fmaxf(fmaf(-gFp, wF, qFf), 0.f), Lf);
+          const float dc = aF * (x - qFf);
+          const float phi = fmaf(dc, fmaf(dc, HFF, gFp), fixed);
+          if (phi <= bound) {
+            const float rFf = rintf(x);
+            const float dF = aF * (rFf - qFf);
+            const float val = fmaf(dF, fmaf(dF, HFF, gFp), fixed);
+            const unsigned r0 = swap ? (unsigned)rFf : (unsigned)rS, r1 = swap ? (unsigned)rS : (unsigned)rFf;
+            const unsigned pk = (m0 << 16) | (r0 << 8) | r1;
+            if (val < best || (val == best && val < 0.f && pk < bpk)) {
+              best = val; bpk = pk; bextra = extra_s;
+              bound = fminf(bound, best);
+            }
+          }
+          return phi;
+        };
+        const float phi_q = eval(qS);
+        float prev = phi_q;
+        for (int rS = qS + 1; rS <= p.L; ++rS) {
+          const float phi = eval(rS);
+          if (!full && phi > bound && phi >= prev) break;
+          prev = phi;
+        }
+        prev = phi_q;
+        for (int rS = qS - 1; rS >= 0; --rS) {
+          const float phi = eval(rS);
+          if (!full && phi > bound && phi >= prev) break;
+          prev = phi;
         }
       }
 
@@ -211,7 +291,6 @@ bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, 
       } else {
         __syncwarp();
       }
-      if (t + 1 < p.T) draw(t + 1);
       if (m == kNoMove) continue;  // this partition holds no improving pair
 
       const unsigned m0 = w >> 16, m1 = extra & 0xFFFFu;
@@ -222,8 +301,8 @@ bcd2_kernel(CdParams p, unsigned long long seed, BcdShape shape, int g_in_smem, 
         bad = true;
         break;
       }
-      const double c0 = 2.0 * ((double)scale_of(m0) * (double)(r0 - q0));
-      const double c1 = 2.0 * ((double)scale_of(m1) * (double)(r1 - q1));
+      const double c0 = 2.0 * ((double)scale_of(m0).x * (double)(r0 - q0));
+      const double c1 = 2.0 * ((double)scale_of(m1).x * (double)(r1 - q1));
       const float* row0 = p.H + (size_t)m0 * d_in;
       const float* row1 = p.H + (size_t)m1 * d_in;
       const unsigned nch = d_in >> 1;
@@ -287,7 +366,7 @@ __global__ void __launch_bounds__(128) bcd2_verify_kernel(CdParams p, unsigned l
   const int nlev = p.L + 1;
   double* g = p.G + j * p.ldg;
   unsigned char* q = p.Qt + j * p.ldq;
-  const unsigned long long base = splitmix64(seed ^ splitmix64((unsigned long long)j));
+  const unsigned long long base = splitmix64(seed);
   unsigned long long moves = 0;
   double dsum = 0.0;
   for (long long t = 0; t < p.T; ++t) {
@@ -366,13 +445,13 @@ bool bcd_supported(long long d_in, int block) {
 }
 
 template <int PPT, int MAXNT, int MINB>
-static cudaError_t launch_bcd_cfg(const CdParams& p, unsigned long long seed, int nt, cudaStream_t st) {
+static cudaError_t launch_bcd_cfg(const CdParams& p, const uint4* tab, int nt, cudaStream_t st) {
   auto kern = bcd2_kernel<PPT, MAXNT, MINB>;
   int dev = 0, sms = 0, smem_max = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  const size_t q_bytes = (size_t)((p.ldg + 15) / 16 * 16), a_bytes = sizeof(float) * (size_t)p.ng;
+  const size_t q_bytes = (size_t)((p.ldg + 15) / 16 * 16), a_bytes = sizeof(float2) * (size_t)p.ng;
   const size_t budget = (size_t)smem_max - 2048;  // the kernel's static shared memory and the runtime's share
   const int a_in_smem = q_bytes + a_bytes <= budget / 2 ? 1 : 0;
   size_t smem = q_bytes + (a_in_smem ? a_bytes : 0);
@@ -392,13 +471,17 @@ static cudaError_t launch_bcd_cfg(const CdParams& p, unsigned long long seed, in
   if (per_sm < 1) return cudaErrorInvalidConfiguration;
   long long blocks = (long long)sms * per_sm;
   if (blocks > p.d_out) blocks = p.d_out;
-  kern<<<(unsigned)blocks, nt, smem, st>>>(p, seed, bcd_shape(p.d_in), g_in_smem, a_in_smem);
+  kern<<<(unsigned)blocks, nt, smem, st>>>(p, tab, g_in_smem, a_in_smem);
   return cudaGetLastError();
 }
 
+size_t bcd_table_bytes(long long d_in, long long steps_per_col) {
+  return sizeof(uint4) * (size_t)(d_in / 2) * (size_t)(steps_per_col > 0 ? steps_per_col : 0);
+}
+
 cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq, const float* hdiag,
-                       const float* hs, long long steps_per_col, unsigned long long seed, bool fast, CdCounters* ctr,
-                       cudaStream_t st) {
+                       const float* hs, long long steps_per_col, unsigned long long seed, bool fast, void* table,
+                       CdCounters* ctr, cudaStream_t st) {
   CdParams p{};
   p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
   p.hdiag = hdiag; p.hs = hs; p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
@@ -410,11 +493,19 @@ cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char*
     return cudaGetLastError();
   }
   const long long nb = ly.d_in / 2;
+  uint4* tab = (uint4*)table;
+  if (steps_per_col > 0) {
+    if (steps_per_col > 65535) return cudaErrorNotSupported;  // steps index a grid dimension
+    dim3 grid((unsigned)((nb + 255) / 256), (unsigned)steps_per_col);
+    bcd2_table_kernel<<<grid, 256, 0, st>>>(ly.H, hdiag, (unsigned)ly.d_in, seed, bcd_shape(ly.d_in), tab);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
   auto team = [&](int ppt) { return (int)(((nb + ppt - 1) / ppt + 31) / 32 * 32); };
-  if (nb <= 256) return launch_bcd_cfg<1, 256, 4>(p, seed, team(1), st);
-  if (nb <= 2048) return launch_bcd_cfg<4, 512, 2>(p, seed, team(4), st);
-  if (nb <= 8192) return launch_bcd_cfg<8, 1024, 1>(p, seed, team(8), st);
-  return launch_bcd_cfg<16, 1024, 1>(p, seed, team(16), st);
+  if (nb <= 256) return launch_bcd_cfg<1, 256, 4>(p, tab, team(1), st);
+  if (nb <= 2048) return launch_bcd_cfg<4, 512, 2>(p, tab, team(4), st);
+  if (nb <= 8192) return launch_bcd_cfg<8, 1024, 1>(p, tab, team(8), st);
+  return launch_bcd_cfg<16, 1024, 1>(p, tab, team(16), st);
 }
 
 }  // namespace cdq

@@ -126,8 +126,9 @@ cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned
 // bcd_kernel.cu: random blocks of two coordinates (Algorithm 2 / 5)
 bool bcd_supported(long long d_in, int block);
 cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq, const float* hdiag,
-                       const float* hs, long long steps_per_col, unsigned long long seed, bool fast, CdCounters* ctr,
-                       cudaStream_t st);
+                       const float* hs, long long steps_per_col, unsigned long long seed, bool fast, void* table,
+                       CdCounters* ctr, cudaStream_t st);
+size_t bcd_table_bytes(long long d_in, long long steps_per_col);  // the production kernel's list of pairs
 cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st);  // ascending order
 cudaError_t launch_sum_f64_tree(const double* v, long long n, double* out, cudaStream_t st);  // fixed tree order
 

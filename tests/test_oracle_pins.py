@@ -433,16 +433,15 @@ def test_owc_cd_against_brute_force_over_all_assignments():
 # ---------------------------------------------------------------- BCD with random blocks (Algorithm 2 / 5)
 def test_bcd_partition_is_a_permutation_and_varies():
     for d in (1, 2, 7, 10, 64, 100, 257):
-        p0 = oracle.bcd_perm(d, 11, 3, 0)
+        p0 = oracle.bcd_perm(d, 11, 0)
         assert sorted(p0.tolist()) == list(range(d))
         if d >= 10:
-            assert not np.array_equal(p0, oracle.bcd_perm(d, 11, 3, 1))      # another step
-            assert not np.array_equal(p0, oracle.bcd_perm(d, 11, 4, 0))      # another column
-            assert not np.array_equal(p0, oracle.bcd_perm(d, 12, 3, 0))      # another seed
+            assert not np.array_equal(p0, oracle.bcd_perm(d, 11, 1))      # another step
+            assert not np.array_equal(p0, oracle.bcd_perm(d, 12, 0))      # another seed
     # every pair of coordinates gets paired at some step: the family is not stuck on a few partitions
     d, seen = 12, set()
     for t in range(400):
-        p = oracle.bcd_perm(d, 5, 0, t)
+        p = oracle.bcd_perm(d, 5, t)
         seen |= {tuple(sorted((int(p[2 * u]), int(p[2 * u + 1])))) for u in range(d // 2)}
     assert len(seen) == d * (d - 1) // 2
 
@@ -468,7 +467,7 @@ def test_bcd_step_is_the_best_block_move_and_loss_is_the_loss_from_x(bits, g, k)
         # brute force over the blocks of pi(., step 0) and all level assignments, loss from the definition
         q0 = init["Q"][:, j].astype(np.int64)
         base = (a[:, j] * q0 + b[:, j] - Wd[:, j]); base = base @ Hd @ base
-        perm = oracle.bcd_perm(d_in, seed, j, 0)
+        perm = oracle.bcd_perm(d_in, seed, 0)
         best, bq = base, q0
         for u in range(d_in // k):
             blk = sorted(int(x) for x in perm[k * u:k * u + k])
