@@ -14,10 +14,10 @@
 // off-diagonal entry H_im (d_in / 2 scattered reads per step, which would otherwise be paid
 // per column and bound the descent by the rate of random DRAM reads) and with the two
 // diagonal entries; the descent reads that table in order (16 bytes per pair and pass).
-// The scan over the (L+1)^2 assignments fixes a level of the lower coordinate and takes the
-// best level of the other in closed form (the clamped rounding of the vertex of its parabola,
-// as in the greedy descent); convexity of the change in the pair bounds which levels of the
-// lower coordinate can still win, so only a few of them are visited.
+// The scan over the (L+1)^2 assignments fixes a level of one coordinate and takes the best
+// level of the other in closed form (the clamped rounding of the vertex of its parabola, as
+// in the greedy descent); convexity of the change in the pair tells which pairs, and which
+// levels, can still win, so only a few are visited (see the kernel's header).
 #include <cstdio>
 #include <cstdlib>
 
@@ -109,24 +109,43 @@ __global__ void bcd2_table_kernel(const float* __restrict__ H, const float* __re
 // PPT: pairs per thread (pair u = tid + NT * slot).  g_in_smem == 0: the gradient stays in
 // its global-memory column (layers whose column does not fit in shared memory).
 // a_in_smem == 0: the group scales are read from global memory.
+//
+// One step:
+//   1. (with the update of the previous step) every thread sweeps its own coordinates, two
+//      per chunk: g += 2 d_i H[i, :] + 2 d_m H[m, :], and the best move of each coordinate
+//      alone is scored as in the greedy descent; its minimum over the team, `bound`, is a
+//      change that some pair reaches (a pair may keep one of its levels);
+//   2. every pair is tested against the bound with the free minimum of its 2 x 2 quadratic,
+//      -N / (4 det), N = g_i^2 H_mm - 2 g_i g_m H_im + g_m^2 H_ii (H is positive
+//      semi-definite, so no assignment of levels does better); most pairs stop here;
+//   3. the pairs that are left are scanned, after the test loop so that a warp scans only as
+//      many rounds as its busiest lane has such pairs: the levels of one coordinate S are
+//      walked outwards from its current level, the level of the other, F, follows in closed
+//      form; phi(r_S), the change with F free in [0, L], is convex in r_S and bounds the
+//      rounded change from below, so a side ends once phi has passed the best change known
+//      and no longer falls.  S is the coordinate with the larger a^2 H_ii (few of its levels
+//      can win).  A pair whose 2 x 2 block is close to singular in fp32 is always scanned, in
+//      full;
+//   4. team-wide argmin (change, lowest first coordinate, lowest levels), as in the greedy
+//      descent, carrying the pair's other coordinate and old levels.
 template <int PPT, int MAXNT, int MINB>
 __global__ void __launch_bounds__(MAXNT, MINB)
 bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_smem) {
   extern __shared__ __align__(16) unsigned char dyn_smem[];
   __shared__ __align__(16) uint4 s_exch[2][32];
-  __shared__ unsigned s_bound[2][32];
+  __shared__ unsigned s_bound[32];
   __shared__ int s_col;
 
   const int tid = threadIdx.x, NT = blockDim.x;
   const int lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
   const unsigned d_in = (unsigned)p.d_in;
-  const unsigned nb = d_in >> 1;
+  const unsigned nb = d_in >> 1;   // pairs, and chunks of two coordinates
   const float Lf = (float)p.L;
 
-  // shared memory: [gradient, 8 ldg bytes][codes, ldg bytes rounded to 16][scales, 4 ng bytes]
+  // shared memory: [gradient, 8 ldg bytes][codes, ldg bytes rounded to 16][(a, 1 / a) per group]
   double* g_smem = reinterpret_cast<double*>(dyn_smem);
   unsigned char* q_s = dyn_smem + (g_in_smem ? sizeof(double) * (size_t)p.ldg : 0);
-  float2* a_smem = reinterpret_cast<float2*>(q_s + ((p.ldg + 15) / 16) * 16);   // (a, 1 / a) per group
+  float2* a_smem = reinterpret_cast<float2*>(q_s + ((p.ldg + 15) / 16) * 16);
   auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
 
   unsigned long long my_moves = 0;
@@ -162,49 +181,86 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
       return make_float2(a, a > 0.f ? 1.0f / a : 0.f);
     };
 
+    // Applies g += c0 row0 + c1 row1 (nrows of them) to the thread's chunks and returns the best
+    // change of a single coordinate among them (0 if none lowers the loss).  A thread owns the
+    // chunks tid + NT * s, s < PPT, as it owns the pairs; the loads of SB chunks are issued
+    // together so that a sweep waits for memory PPT / SB times, not once per chunk.
+    auto sweep = [&](int nrows, double c0, double c1, const float* row0, const float* row1) -> float {
+      constexpr int SB = PPT < 4 ? PPT : 4;
+      float ub = 0.f;
+#pragma unroll
+      for (int s0 = 0; s0 < PPT; s0 += SB) {
+        float2 ha[SB], hb[SB], hd[SB], hs[SB];
+#pragma unroll
+        for (int k = 0; k < SB; ++k) {
+          const unsigned c = (unsigned)tid + (unsigned)NT * (s0 + k);
+          ha[k] = hb[k] = hd[k] = hs[k] = make_float2(0.f, 0.f);
+          if (c < nb) {
+            if (nrows >= 1) ha[k] = ld_row2(row0 + 2 * c);
+            if (nrows == 2) hb[k] = ld_row2(row1 + 2 * c);
+            hd[k] = __ldg(reinterpret_cast<const float2*>(p.hdiag) + c);
+            hs[k] = __ldg(reinterpret_cast<const float2*>(p.hs) + c);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < SB; ++k) {
+          const unsigned c = (unsigned)tid + (unsigned)NT * (s0 + k);
+          if (c >= nb) continue;
+          double2 gv = *reinterpret_cast<double2*>(g_s + 2 * c);
+          if (nrows >= 1) {
+            gv.x = fma(c0, (double)ha[k].x, gv.x);
+            gv.y = fma(c0, (double)ha[k].y, gv.y);
+          }
+          if (nrows == 2) {
+            gv.x = fma(c1, (double)hb[k].x, gv.x);
+            gv.y = fma(c1, (double)hb[k].y, gv.y);
+          }
+          if (nrows >= 1) *reinterpret_cast<double2*>(g_s + 2 * c) = gv;
+          const unsigned qq = *reinterpret_cast<const unsigned short*>(q_s + 2 * c);
+          const float2 ax = scale_of(2 * c), ay = scale_of(2 * c + 1);
+          {
+            const float gf = (float)gv.x, qf = (float)(qq & 255u);
+            const float rf = fminf(fmaxf(rintf(fmaf(-gf, hs[k].x * ax.y, qf)), 0.f), Lf);
+            const float d = ax.x * (rf - qf);
+            ub = fminf(ub, d * fmaf(d, hd[k].x, gf));
+          }
+          {
+            const float gf = (float)gv.y, qf = (float)(qq >> 8);
+            const float rf = fminf(fmaxf(rintf(fmaf(-gf, hs[k].y * ay.y, qf)), 0.f), Lf);
+            const float d = ay.x * (rf - qf);
+            ub = fminf(ub, d * fmaf(d, hd[k].y, gf));
+          }
+        }
+      }
+      return ub;
+    };
+    // Team-wide minimum of the sweeps' results; ends with every thread past the barrier.
+    auto team_bound = [&](float ub) -> float {
+      unsigned k = __reduce_min_sync(0xFFFFFFFFu, ub < 0.f ? ~__float_as_uint(ub) : kNoMove);
+      if (nwarps > 1) {
+        if (lane == 0) s_bound[warp] = k;
+        __syncthreads();
+        k = __reduce_min_sync(0xFFFFFFFFu, lane < nwarps ? s_bound[lane] : kNoMove);
+      } else {
+        __syncwarp();
+      }
+      return k == kNoMove ? 0.f : __uint_as_float(~k);
+    };
+
     double col_dsum = 0.0;
     long long moves = 0;
     bool bad = false;
+    float bound = p.T > 0 ? team_bound(sweep(0, 0.0, 0.0, p.H, p.H)) : 0.f;
     for (long long t = 0; t < p.T; ++t) {
-      // ---- pass 1: the best move of each coordinate alone (the pair with the other level kept) ----
       const uint4* trow = tab + (size_t)t * nb;
+      // what a pair has to reach: the bound, eased by a few ulps so that the single move that
+      // set it is found again by the scan of its pair
+      float lim = bound * 0.99999f;
       float best = 0.f;
       unsigned bpk = kNoMove, bextra = 0;
-#pragma unroll
-      for (int s = 0; s < PPT; ++s) {
-        const unsigned u = (unsigned)tid + (unsigned)NT * s;
-        if (u >= nb) continue;
-        const uint4 e = __ldg(trow + u);
-        const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
-        const unsigned q0 = q_s[m0], q1 = q_s[m1];
-        const unsigned extra_s = m1 | (q0 << 16) | (q1 << 24);
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          const unsigned mc = c ? m1 : m0;
-          const float gc = (float)g_s[mc], qf = (float)(c ? q1 : q0);
-          const float2 ac = scale_of(mc);
-          const float Hcc = __uint_as_float(c ? e.w : e.z);
-          const float hsc = Hcc > 0.f ? 0.5f / Hcc : 0.f;
-          const float rf = fminf(fmaxf(rintf(fmaf(-gc, hsc * ac.y, qf)), 0.f), Lf);
-          const float d = ac.x * (rf - qf);
-          const float val = d * fmaf(d, Hcc, gc);
-          const unsigned pk = (m0 << 16) | (c ? (q0 << 8) | (unsigned)rf : ((unsigned)rf << 8) | q1);
-          if (val < best || (val == best && val < 0.f && pk < bpk)) { best = val; bpk = pk; bextra = extra_s; }
-        }
-      }
-      // the best of them over the team bounds what a pair has to beat
-      float bound;
-      {
-        unsigned k1 = __reduce_min_sync(0xFFFFFFFFu, best < 0.f ? ~__float_as_uint(best) : kNoMove);
-        if (nwarps > 1) {
-          if (lane == 0) s_bound[xbuf][warp] = k1;
-          __syncthreads();
-          k1 = __reduce_min_sync(0xFFFFFFFFu, lane < nwarps ? s_bound[xbuf][lane] : kNoMove);
-        }
-        bound = k1 == kNoMove ? 0.f : __uint_as_float(~k1);
-      }
 
-      // ---- pass 2: pairs that can beat the bound ----
+      // ---- test every pair of this thread against the bound ----
+      unsigned todo = 0;
 #pragma unroll
       for (int s = 0; s < PPT; ++s) {
         const unsigned u = (unsigned)tid + (unsigned)NT * s;
@@ -213,20 +269,26 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
         const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
         const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
         const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
-        const float h2 = 2.f * h01;
-        // The change is convex in the pair (H is positive semi-definite): no assignment does
-        // better than the free minimum -N / (4 det), N = g0^2 H11 - 2 g0 g1 H01 + g1^2 H00.
-        // A pair whose 2 x 2 block of H is close to singular in fp32 is never skipped and is
-        // scanned in full.
         const float det = fmaf(H00, H11, -h01 * h01);
+        const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
         const bool full = !(det > 1e-4f * H00 * H11);
-        const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -g0 * g1 * h2));
-        if (!full && 1.001f * N < -4.f * bound * det) continue;
+        if (full || !(1.01f * N < -4.f * lim * det)) todo |= 1u << s;   // 1 % for the rounding of N and det
+      }
+
+      // ---- scan the pairs that are left ----
+      while (todo) {
+        const int s = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const unsigned u = (unsigned)tid + (unsigned)NT * s;
+        const uint4 e = __ldg(trow + u);
+        const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
+        const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
+        const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
+        const float h2 = 2.f * h01;
+        const bool full = !(fmaf(H00, H11, -h01 * h01) > 1e-4f * H00 * H11);
         const int q0 = q_s[m0], q1 = q_s[m1];
         const float2 a0 = scale_of(m0), a1 = scale_of(m1);
         const unsigned extra_s = m1 | ((unsigned)q0 << 16) | ((unsigned)q1 << 24);
-        // S: the coordinate whose levels are scanned (the one with the larger a^2 H_ii, so that
-        // few of its levels can win); F: the other, whose level follows in closed form
         const bool swap = !full && a1.x * a1.x * H11 > a0.x * a0.x * H00;
         const float gS = swap ? g1 : g0, gF = swap ? g0 : g1;
         const int qS = swap ? q1 : q0, qF = swap ? q0 : q1;
@@ -234,9 +296,6 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
         const float HSS = swap ? H11 : H00, HFF = swap ? H00 : H11;
         const float wF = HFF > 0.f ? 0.5f / HFF * (swap ? a0.y : a1.y) : 0.f;   // 1 / (2 a H_ii)
         const float qFf = (float)qF;
-        // phi(rS): the change with F free in [0, L] (not rounded): convex in rS and a lower
-        // bound of the rounded change, so the scan walks outwards from qS and stops on a side
-        // once phi has passed the bound and no longer falls.
         auto eval = [&](int rS) -> float {
           const float dS = aS * (float)(rS - qS);
           const float fixed = dS * fmaf(dS, HSS, gS);
@@ -244,7 +303,7 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
           const float x = fminf(fmaxf(fmaf(-gFp, wF, qFf), 0.f), Lf);
           const float dc = aF * (x - qFf);
           const float phi = fmaf(dc, fmaf(dc, HFF, gFp), fixed);
-          if (phi <= bound) {
+          if (phi <= lim) {
             const float rFf = rintf(x);
             const float dF = aF * (rFf - qFf);
             const float val = fmaf(dF, fmaf(dF, HFF, gFp), fixed);
@@ -252,7 +311,7 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
             const unsigned pk = (m0 << 16) | (r0 << 8) | r1;
             if (val < best || (val == best && val < 0.f && pk < bpk)) {
               best = val; bpk = pk; bextra = extra_s;
-              bound = fminf(bound, best);
+              lim = fminf(lim, best * 0.99999f);
             }
           }
           return phi;
@@ -261,13 +320,13 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
         float prev = phi_q;
         for (int rS = qS + 1; rS <= p.L; ++rS) {
           const float phi = eval(rS);
-          if (!full && phi > bound && phi >= prev) break;
+          if (!full && phi > lim && phi >= prev) break;
           prev = phi;
         }
         prev = phi_q;
         for (int rS = qS - 1; rS >= 0; --rS) {
           const float phi = eval(rS);
-          if (!full && phi > bound && phi >= prev) break;
+          if (!full && phi > lim && phi >= prev) break;
           prev = phi;
         }
       }
@@ -291,7 +350,7 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
       } else {
         __syncwarp();
       }
-      if (m == kNoMove) continue;  // this partition holds no improving pair
+      if (m == kNoMove) continue;  // this partition holds no improving pair; the state and the bound stand
 
       const unsigned m0 = w >> 16, m1 = extra & 0xFFFFu;
       const int r0 = (int)((w >> 8) & 255u), r1 = (int)(w & 255u);
@@ -305,35 +364,19 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
       const double c1 = 2.0 * ((double)scale_of(m1).x * (double)(r1 - q1));
       const float* row0 = p.H + (size_t)m0 * d_in;
       const float* row1 = p.H + (size_t)m1 * d_in;
-      const unsigned nch = d_in >> 1;
-      if (c0 != 0.0 && c1 != 0.0) {
-#pragma unroll 4
-        for (unsigned c = tid; c < nch; c += NT) {
-          const float2 ha = ld_row2(row0 + 2 * c), hb = ld_row2(row1 + 2 * c);
-          double2 gv = *reinterpret_cast<double2*>(g_s + 2 * c);
-          gv.x = fma(c1, (double)hb.x, fma(c0, (double)ha.x, gv.x));
-          gv.y = fma(c1, (double)hb.y, fma(c0, (double)ha.y, gv.y));
-          *reinterpret_cast<double2*>(g_s + 2 * c) = gv;
-        }
-      } else {
-        const float* row = c0 != 0.0 ? row0 : row1;
-        const double cc = c0 != 0.0 ? c0 : c1;
-#pragma unroll 4
-        for (unsigned c = tid; c < nch; c += NT) {
-          const float2 ha = ld_row2(row + 2 * c);
-          double2 gv = *reinterpret_cast<double2*>(g_s + 2 * c);
-          gv.x = fma(cc, (double)ha.x, gv.x);
-          gv.y = fma(cc, (double)ha.y, gv.y);
-          *reinterpret_cast<double2*>(g_s + 2 * c) = gv;
-        }
-      }
+      // the new codes are written by the threads that own these coordinates in the sweep, the
+      // only readers of a code until the barrier that ends it
+      if ((unsigned)tid == (m0 >> 1) % (unsigned)NT) q_s[m0] = (unsigned char)r0;
+      if ((unsigned)tid == (m1 >> 1) % (unsigned)NT) q_s[m1] = (unsigned char)r1;
+      float ub;
+      if (c0 != 0.0 && c1 != 0.0) ub = sweep(2, c0, c1, row0, row1);
+      else if (c0 != 0.0) ub = sweep(1, c0, 0.0, row0, row0);
+      else ub = sweep(1, c1, 0.0, row1, row1);
       if (tid == 0) {
-        q_s[m0] = (unsigned char)r0;
-        q_s[m1] = (unsigned char)r1;
         col_dsum += (double)__uint_as_float(~m);
         ++moves;
       }
-      __syncthreads();
+      bound = team_bound(ub);
     }
     if (tid == 0) { my_moves += (unsigned long long)moves; my_dsum += col_dsum; }
     __syncthreads();
@@ -502,8 +545,9 @@ cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char*
     if (e != cudaSuccess) return e;
   }
   auto team = [&](int ppt) { return (int)(((nb + ppt - 1) / ppt + 31) / 32 * 32); };
-  if (nb <= 256) return launch_bcd_cfg<1, 256, 4>(p, tab, team(1), st);
+  if (nb <= 256) return launch_bcd_cfg<1, 256, 2>(p, tab, team(1), st);
   if (nb <= 2048) return launch_bcd_cfg<4, 512, 2>(p, tab, team(4), st);
+  if (nb <= 7168) return launch_bcd_cfg<8, 896, 1>(p, tab, team(8), st);
   if (nb <= 8192) return launch_bcd_cfg<8, 1024, 1>(p, tab, team(8), st);
   return launch_bcd_cfg<16, 1024, 1>(p, tab, team(16), st);
 }
