@@ -170,6 +170,9 @@ def main():
     ap.add_argument("--init", default="rtn", choices=["rtn", "owc_cd"],
                     help="grid stage: cdq_init_rtn (MinMax / OWC as the config says) or cdq_init_owc_cd (Algorithm 3; "
                          "configs with a clipping grid)")
+    ap.add_argument("--shard", action="store_true",
+                    help="share ONE layer out over the ranks (strong scaling): rows of X per rank for the Hessian with one "
+                         "all-reduce, columns of W per rank after it; the default gives every rank its own layer (weak)")
     ap.add_argument("--d-out", type=int, default=0, help="profiling case: keep only this many output columns")
     ap.add_argument("--n", type=int, default=0, help="profiling case: keep only this many calibration rows")
     args = ap.parse_args()
@@ -205,8 +208,12 @@ def main():
 
     # every rank quantizes its own layer (same shape, its own seed): columns and layers are
     # independent problems, so there is no data-path collective
-    my_cfg = cfg.scaled(seed=multi.rank_seed(cfg.seed, rank))
+    my_cfg = cfg if args.shard else cfg.scaled(seed=multi.rank_seed(cfg.seed, rank))
     X, W = inputs.make_layer(my_cfg, device=dev)
+    if args.shard:   # the same layer everywhere; this rank keeps its rows of X and its columns of W
+        r0, r1 = multi.shard_range(cfg.n, world, rank, multiple=64)
+        c0, c1 = multi.shard_range(cfg.d_out, world, rank)
+        X, W = X[r0:r1].contiguous(), W[:, c0:c1].contiguous()
     Xh, Wh = X.cpu().pin_memory(), W.cpu().pin_memory()
     grid = B.Grid(cfg.bits, cfg.group_size, cfg.n_clip, cfg.clip_lo, cfg.clip_hi)
     ws = B.Workspace()
@@ -222,6 +229,8 @@ def main():
         Wd = Wh.to(dev, non_blocking=True) if host else W
         ev[1].record()
         H = B.cdq_hessian(Xd, ws=ws)
+        if args.shard and world > 1:   # the one exchange of the sharded layer: sum of the row shards' Hessians
+            dist.all_reduce(H, op=dist.ReduceOp.SUM)
         ev[2].record()
         if args.init == "owc_cd":
             scale, zero, Q, _, _ = B.cdq_init_owc_cd(Wd, grid, H, ws=ws)
@@ -283,29 +292,31 @@ def main():
         return
 
     peaks = load_peaks()
+    acc = cfg.scaled(d_out=W.shape[1], n=X.shape[0])   # what this rank worked on (the whole layer unless --shard)
     ms_per_step = total_ms / args.steps
     value = multi.whole_job_throughput(committed_all, total_ms, args.steps)
     mean = lambda v: sum(v) / len(v)
     cd_ms = mean(times["cd_kernel"])
-    alg_bytes = algorithmic_bytes_cd(cfg, committed)
+    alg_bytes = algorithmic_bytes_cd(acc, committed)
     if args.block == 2:  # two rows per move at most, and one H_im per pair and step
         alg_bytes += committed * 4.0 * cfg.d_in + stats["steps"] * 2.0 * cfg.d_in
     achieved = alg_bytes / (cd_ms * 1e-3) / 1e9
     h_in_l2 = 4.0 * cfg.d_in * cfg.d_in < 100e6
     hess_ms = mean(times["hessian"])
-    hess_flops = 2.0 * cfg.n * cfg.d_in * cfg.d_in
+    hess_flops = 2.0 * acc.n * cfg.d_in * cfg.d_in
     # flops the tensor cores actually execute: 128 x 256 tiles that touch the lower triangle
     # (tile (tm, tn) with tn <= tm // 2), over the rows padded to the 64-row K block
     tiles_m = (cfg.d_in + 127) // 128
     n_tiles = sum(tm // 2 + 1 for tm in range(tiles_m))
-    hess_exec = 2.0 * 128 * 256 * n_tiles * ((cfg.n + 63) // 64 * 64) if cfg.x_dtype == "bf16" and cfg.d_in >= 256 else hess_flops
+    hess_exec = 2.0 * 128 * 256 * n_tiles * ((acc.n + 63) // 64 * 64) if cfg.x_dtype == "bf16" and cfg.d_in >= 256 else hess_flops
     h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if args.shard else "weak", "vs_baseline": None,
         "dtype": "f32 scores / f64 gradient / bf16 Hessian inputs", "data": "synthetic",
         "config": {"workload": workload, "l2": "256 MiB flush between timed iterations; X also exceeds L2",
-                   "per_rank": "one independent layer per GPU, no collective"},
+                   "per_rank": ("one layer shared out: row shards of X + one all-reduce of H, column slices of W after it"
+                                if args.shard else "one independent layer per GPU, no collective")},
         "sec_per_layer": ms_per_step * 1e-3,
         "cd": {"committed_updates": committed, "step_budget": stats["steps"],
                "columns_converged": stats["columns_converged"], "kernel_ms": cd_ms,
@@ -328,7 +339,7 @@ def main():
                               if h_in_l2 else "H exceeds L2: rows stream from HBM")},
         "e2e": {"value": committed_all / (total_ms_e2e / args.steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": total_ms_e2e / args.steps},
-        "gpu_launches": kernel_launches(cfg) * args.steps,
+        "gpu_launches": kernel_launches(acc) * args.steps,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline and args.block == 1:

@@ -109,6 +109,15 @@ cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in,
                        size_t ws_bytes, void* stream);
 
 /*
+ * The regulariser alone: H_ii += lambda_rel * mean(diag H) (paper: Section 4, "we regularize the
+ * Hessian ... by adding lambda I").  For a Hessian that is summed from several parts first (row
+ * chunks, or the row shards of several GPUs after their all-reduce): the parts are formed with
+ * lambda_rel = 0 and the sum is regularised once.
+ *   H  [d_in, d_in] fp32 device, in/out.  lambda_rel >= 0.
+ */
+cdq_status cdq_hessian_add_lambda(float* H, long long d_in, float lambda_rel, void* stream);
+
+/*
  * Grid and round-to-nearest codes (paper: Eq. 2; gamma = 1 is MinMax), with
  * the Optimal Weight Clipping search when grid->n_clip > 1 (paper: the
  * minimisation over gamma stated after Eq. 2, solved by grid search).

@@ -24,7 +24,7 @@ MODE_FAST, MODE_FP64_VERIFY = 0, 1
 CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD, CALL_BCD_SOLVE = 0, 1, 2, 3, 4, 5
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
+EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version"]
 
@@ -89,6 +89,8 @@ def load():
                                     ci, vp, sz, vp]
     lib.cdq_cd_solve.restype = ci
     lib.cdq_cd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
+    lib.cdq_hessian_add_lambda.restype = ci
+    lib.cdq_hessian_add_lambda.argtypes = [vp, ll, ctypes.c_float, vp]
     lib.cdq_bcd_solve.restype = ci
     lib.cdq_bcd_solve.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ci, ll, ctypes.c_ulonglong, ci,
                                   ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
@@ -164,6 +166,14 @@ def cdq_hessian(X: torch.Tensor, lambda_rel: float = 0.0, accumulate: bool = Fal
     st = load().cdq_hessian(X.data_ptr(), _dtype_code(X), n, d_in, X.stride(0), float(lambda_rel), int(accumulate),
                             H.data_ptr(), _MODES[mode], wptr, wbytes, _stream())
     _check(st, "cdq_hessian")
+    return H
+
+
+def cdq_hessian_add_lambda(H: torch.Tensor, lambda_rel: float) -> torch.Tensor:
+    """H_ii += lambda_rel * mean(diag H), in place (for a Hessian summed from parts)."""
+    _need_cuda(H)
+    assert H.dim() == 2 and H.shape[0] == H.shape[1] and H.is_contiguous() and H.dtype == torch.float32
+    _check(load().cdq_hessian_add_lambda(H.data_ptr(), H.shape[0], float(lambda_rel), _stream()), "cdq_hessian_add_lambda")
     return H
 
 

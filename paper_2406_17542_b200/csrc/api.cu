@@ -233,6 +233,14 @@ cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in,
   return CDQ_OK;
 }
 
+cdq_status cdq_hessian_add_lambda(float* H, long long d_in, float lambda_rel, void* stream) {
+  if (!H || !(lambda_rel >= 0.f)) return CDQ_ERR_INVALID_ARG;
+  if (d_in < 1) return CDQ_ERR_SHAPE;
+  if (d_in > 65535) return CDQ_ERR_UNSUPPORTED;
+  if (lambda_rel > 0.f) CDQ_CUDA(launch_hessian_lambda(H, d_in, (double)lambda_rel, nullptr, (cudaStream_t)stream));
+  return CDQ_OK;
+}
+
 cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw, const float* H,
                         const cdq_grid_desc* grid, float* scale, float* zero, unsigned char* Q, float* gamma_out,
                         cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {

@@ -188,3 +188,22 @@ def test_reduced_step_budget(mode, frac):
     else:
         assert float((Q.cpu().numpy() == ref["Q"]).mean()) >= CODE_AGREE
         np.testing.assert_allclose(st["loss_after"], ref["loss_after"], rtol=LOSS_RTOL)
+
+
+def test_regulariser_alone_matches_the_fused_one():
+    """cdq_hessian_add_lambda on a Hessian summed from row chunks == cdq_hessian with lambda_rel (Section 4)."""
+    cfg = inputs.CONFIGS["C0"].scaled(d_in=320, n=1536, x_dtype="bf16", seed=77)
+    X = inputs.make_x(cfg, device="cuda:0")
+    fused = B.cdq_hessian(X, lambda_rel=0.01)
+    parts = B.cdq_hessian(X[:1024].contiguous())
+    B.cdq_hessian(X[1024:].contiguous(), accumulate=True, out=parts)
+    plain = parts.clone()
+    B.cdq_hessian_add_lambda(parts, 0.01)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(parts.cpu().numpy(), fused.cpu().numpy(), rtol=1e-5, atol=1e-5 * float(fused.abs().max()))
+    add = (parts.diagonal() - plain.diagonal()).double()
+    # the sum is rounded to fp32: each entry is off by up to half an ulp of H_ii
+    np.testing.assert_allclose(add.cpu().numpy(), 0.01 * float(plain.diagonal().double().mean()), rtol=1e-4,
+                               atol=1.2e-7 * float(plain.diagonal().max()))
+    off = ~torch.eye(cfg.d_in, dtype=torch.bool, device="cuda:0")
+    assert torch.equal(parts[off], plain[off])
