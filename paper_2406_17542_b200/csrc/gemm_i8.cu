@@ -30,7 +30,8 @@ namespace i8 {
 constexpr int BM = 128, BN = 256, BKB = 128;       // tile; BKB = bytes (= int8 elements) of K per stage
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BKB, B_BYTES = BN * BKB, STAGE_BYTES = A_BYTES + B_BYTES;  // 16 + 32 KB
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;     // producer, MMA issuer, 8 epilogue warps (two per TMEM lane quarter)
+constexpr int EPI_WARPS = 8;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
 constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 256;
@@ -141,6 +142,9 @@ struct Params {
   const int* eexp;          // [M]
   const int* hexp;          // [N]
   double final_scale;       // applied with the exponents after the last group
+  const double* E;          // optional, [N, lde]: with dot_part, the epilogue also sums E[p, j] C[j, p] over its columns
+  long long lde;
+  double* dot_part;         // [2 * tiles_n, M] partial column dots, one row per (tile column, epilogue half)
   int* status;
 };
 
@@ -239,7 +243,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_e, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -327,7 +331,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_e, const __grid_constant_
     }
   } else {
     // ---------------- epilogue: TMEM -> fp64 running sum in C ----------------
+    // Two warps per TMEM lane quarter; they take the 16-column chunks of the tile in turn.
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;       // which of the two warps of the quarter
     const int row = q * 32 + lane;          // row of the tile
     int buf = 0;
     uint32_t tphase = 0;
@@ -340,25 +346,54 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_e, const __grid_constant_
       const bool row_ok = j < p.M;
       double* crow = p.C + (row_ok ? j : 0) * p.ldc;
       const int ej = row_ok ? p.eexp[j] : 0;
+      double dot = 0.0;
       for (int g = 0; g < p.ngroups && ok; ++g) {
         if (!mbar_wait(tfull_bar(buf), tphase, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const double w = ldexp(1.0, -7 * p.group_s[g]);
         const bool first = g == 0, last = g == p.ngroups - 1;
 #pragma unroll 1
-        for (int c = 0; c < BN / 16; ++c) {
+        for (int c = half; c < BN / 16; c += 2) {
           uint32_t r[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 16), r);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
           if (row_ok) {
+            const long long pc0 = p0 + c * 16;
+            if (pc0 + 16 <= p.N) {
+              // whole chunk inside the matrix: 16-byte accesses (ldc is a multiple of 4, pc0 of 16)
+              double2* cp = reinterpret_cast<double2*>(crow + pc0);
+              double2 old[8];
+              if (!first) {
 #pragma unroll
-            for (int v = 0; v < 16; ++v) {
-              const long long pc = p0 + c * 16 + v;
-              if (pc < p.N) {
-                double x = w * (double)(int)r[v];
-                if (!first) x += crow[pc];
-                if (last) x = ldexp(x * p.final_scale, ej + p.hexp[pc]);
-                crow[pc] = x;
+                for (int v = 0; v < 8; ++v) old[v] = cp[v];
+              }
+#pragma unroll
+              for (int v = 0; v < 8; ++v) {
+                double x0 = w * (double)(int)r[2 * v], x1 = w * (double)(int)r[2 * v + 1];
+                if (!first) { x0 += old[v].x; x1 += old[v].y; }
+                if (last) {
+                  x0 = ldexp(x0 * p.final_scale, ej + p.hexp[pc0 + 2 * v]);
+                  x1 = ldexp(x1 * p.final_scale, ej + p.hexp[pc0 + 2 * v + 1]);
+                  if (p.dot_part) {
+                    dot = fma(p.E[(pc0 + 2 * v) * p.lde + j], x0, dot);
+                    dot = fma(p.E[(pc0 + 2 * v + 1) * p.lde + j], x1, dot);
+                  }
+                }
+                cp[v] = make_double2(x0, x1);
+              }
+            } else {
+#pragma unroll
+              for (int v = 0; v < 16; ++v) {
+                const long long pc = pc0 + v;
+                if (pc < p.N) {
+                  double x = w * (double)(int)r[v];
+                  if (!first) x += crow[pc];
+                  if (last) {
+                    x = ldexp(x * p.final_scale, ej + p.hexp[pc]);
+                    if (p.dot_part) dot = fma(p.E[pc * p.lde + j], x, dot);
+                  }
+                  crow[pc] = x;
+                }
               }
             }
           }
@@ -368,6 +403,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_e, const __grid_constant_
         if (lane == 0) mbar_arrive(tempty_bar(buf));
         if (++buf == 2) { buf = 0; tphase ^= 1u; }
       }
+      if (p.dot_part && row_ok && ok) p.dot_part[(size_t)(2 * tn + half) * p.M + j] = dot;
     }
   }
 
@@ -381,34 +417,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_e, const __grid_constant_
   }
 }
 
-// col_loss[j] = inv_scale * sum_p E[p, j] * C[j, p]  (fixed summation order: deterministic).
-__global__ void __launch_bounds__(256) coldot_kernel(const double* __restrict__ E, const double* __restrict__ C,
-                                                     long long ldc, long long d_in, long long d_out, double inv_scale,
-                                                     double* __restrict__ col_loss) {
-  __shared__ double tile[32][33];
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const long long j0 = (long long)blockIdx.x * 32;
-  double acc[4] = {0.0, 0.0, 0.0, 0.0};
-  for (long long p0 = 0; p0 < d_in; p0 += 32) {
-    for (int rr = w; rr < 32; rr += 8) {
-      const long long pp = p0 + rr, j = j0 + lane;
-      tile[rr][lane] = (pp < d_in && j < d_out) ? E[pp * d_out + j] : 0.0;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const long long j = j0 + 4 * w + c, pp = p0 + lane;
-      if (j < d_out && pp < d_in) acc[c] = fma(tile[lane][4 * w + c], C[j * ldc + pp], acc[c]);
-    }
-    __syncthreads();
-  }
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    double v = acc[c];
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    const long long j = j0 + 4 * w + c;
-    if (lane == 0 && j < d_out) col_loss[j] = v * inv_scale;
-  }
+// col_loss[j] = inv_scale * sum_b part[b, j], b ascending: the partial column dots
+// sum_p E[p, j] C[j, p] that the GEMM's epilogue leaves per (tile column, epilogue half).  The
+// order of the sum is fixed, so the result does not depend on the schedule.
+__global__ void __launch_bounds__(256) dot_reduce_kernel(const double* __restrict__ part, int nparts, long long m,
+                                                         double inv_scale, double* __restrict__ col_loss) {
+  const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= m) return;
+  double v = 0.0;
+  for (int b = 0; b < nparts; ++b) v += part[(size_t)b * m + j];
+  col_loss[j] = v * inv_scale;
 }
 
 }  // namespace i8
@@ -427,7 +445,8 @@ size_t gemm_tc_h_bytes(long long d_in, int nh) {
   return align_up((size_t)nh * d_in * tc_kpad(d_in)) + align_up(sizeof(int) * (size_t)d_in);
 }
 size_t gemm_tc_e_bytes(long long d_in, long long d_out, int ne) {
-  return align_up((size_t)ne * d_out * tc_kpad(d_in)) + align_up(sizeof(int) * (size_t)d_out) +
+  return align_up(sizeof(double) * 2 * (size_t)((d_in + i8::BN - 1) / i8::BN) * (size_t)d_out) +   // partial column dots
+         align_up((size_t)ne * d_out * tc_kpad(d_in)) + align_up(sizeof(int) * (size_t)d_out) +
          align_up(sizeof(unsigned long long) * (size_t)d_out);
 }
 
@@ -478,6 +497,7 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
   signed char* esl = (signed char*)ebuf;
   int* eexp = (int*)((char*)ebuf + align_up((size_t)ne * d_out * kp));
   unsigned long long* colmax = (unsigned long long*)((char*)eexp + align_up(sizeof(int) * (size_t)d_out));
+  double* dot_part = (double*)((char*)colmax + align_up(sizeof(unsigned long long) * (size_t)d_out));
 
   cudaError_t e = cudaMemsetAsync(colmax, 0, sizeof(unsigned long long) * (size_t)d_out, st);
   if (e != cudaSuccess) return e;
@@ -508,6 +528,7 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
   p.group_first[ng] = npairs;
   p.ngroups = ng;
   p.C = C; p.ldc = ldc; p.eexp = eexp; p.hexp = hexp; p.final_scale = scale;
+  p.E = E; p.lde = d_out; p.dot_part = col_loss ? dot_part : nullptr;
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
 
@@ -526,7 +547,7 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (col_loss) {
-    coldot_kernel<<<(unsigned)((d_out + 31) / 32), 256, 0, st>>>(E, C, ldc, d_in, d_out, 1.0 / scale, col_loss);
+    dot_reduce_kernel<<<(unsigned)((d_out + 255) / 256), 256, 0, st>>>(dot_part, 2 * p.tiles_n, d_out, 1.0 / scale, col_loss);
     e = cudaGetLastError();
   }
   return e;
