@@ -222,6 +222,8 @@ def main():
     def barrier():
         multi.barrier(world)
 
+    pinned_out: list = []
+
     def one_step(host: bool, times: dict | None = None):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
         ev[0].record()
@@ -247,9 +249,13 @@ def main():
             stats["loss_after_cd"] = cd_stats["loss_after"]
         ev[4].record()
         loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws)
-        if host:
-            out = (Q.cpu(), scale.cpu(), zero.cpu())
-            d2h = sum(t.numel() * t.element_size() for t in out) + 8
+        if host:   # results back into pinned host buffers (allocated once, reused every step)
+            srcs = (Q, scale, zero)
+            if not pinned_out:
+                pinned_out.extend(torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in srcs)
+            for dst, src in zip(pinned_out, srcs):
+                dst.copy_(src, non_blocking=True)
+            d2h = sum(t.numel() * t.element_size() for t in srcs) + 8
         else:
             d2h = 0
         ev[5].record()
