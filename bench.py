@@ -109,7 +109,7 @@ def kernel_launches(cfg) -> int:
     tc_g = cfg.d_in >= 256 and cfg.d_out >= 128                                  # int8 tensor-core H E
     hessian = 3 if tc_h else 1
     prep_h = 2                                                                   # row exponents, slices of H
-    he = 5 if tc_g else 2                # column max, exponents, slices of E^T, GEMM, column dot | GEMM, partial sums
+    he = 5 if tc_g else 2                # column max, exponents, slices of E^T, GEMM, sum of the column dots | GEMM, partial sums
     init = 5                                                                     # min/max x2, gamma fill or argmin, scale/zero, codes
     if cfg.n_clip > 1:
         init += (prep_h if tc_g else 0) + cfg.n_clip * (1 + he)                  # per gamma: residual + H E

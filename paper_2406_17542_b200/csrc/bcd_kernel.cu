@@ -175,7 +175,14 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
         a_smem[t] = make_float2(a, a > 0.f ? 1.0f / a : 0.f);
       }
     __syncthreads();
+    const bool one_scale = p.ng == 1;   // per-channel grid: one (a, 1 / a) for the column
+    float2 a_col = make_float2(0.f, 0.f);
+    if (one_scale) {
+      const float a = p.scale[j];
+      a_col = make_float2(a, a > 0.f ? 1.0f / a : 0.f);
+    }
     auto scale_of = [&](unsigned i) -> float2 {
+      if (one_scale) return a_col;
       if (a_in_smem) return a_smem[group_of(i)];
       const float a = p.scale[(long long)group_of(i) * p.d_out + j];
       return make_float2(a, a > 0.f ? 1.0f / a : 0.f);
@@ -259,30 +266,10 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
       float best = 0.f;
       unsigned bpk = kNoMove, bextra = 0;
 
-      // ---- test every pair of this thread against the bound ----
-      unsigned todo = 0;
-#pragma unroll
-      for (int s = 0; s < PPT; ++s) {
-        const unsigned u = (unsigned)tid + (unsigned)NT * s;
-        if (u >= nb) continue;
-        const uint4 e = __ldg(trow + u);
+      // Scan of one pair: the levels of S outwards from its current level, the level of F in
+      // closed form (see the header of the kernel).
+      auto scan_pair = [&](const uint4 e, const float g0, const float g1) {
         const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
-        const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
-        const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
-        const float det = fmaf(H00, H11, -h01 * h01);
-        const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
-        const bool full = !(det > 1e-4f * H00 * H11);
-        if (full || !(1.01f * N < -4.f * lim * det)) todo |= 1u << s;   // 1 % for the rounding of N and det
-      }
-
-      // ---- scan the pairs that are left ----
-      while (todo) {
-        const int s = __ffs(todo) - 1;
-        todo &= todo - 1;
-        const unsigned u = (unsigned)tid + (unsigned)NT * s;
-        const uint4 e = __ldg(trow + u);
-        const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
-        const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
         const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
         const float h2 = 2.f * h01;
         const bool full = !(fmaf(H00, H11, -h01 * h01) > 1e-4f * H00 * H11);
@@ -294,7 +281,7 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
         const int qS = swap ? q1 : q0, qF = swap ? q0 : q1;
         const float aS = swap ? a1.x : a0.x, aF = swap ? a0.x : a1.x;
         const float HSS = swap ? H11 : H00, HFF = swap ? H00 : H11;
-        const float wF = HFF > 0.f ? 0.5f / HFF * (swap ? a0.y : a1.y) : 0.f;   // 1 / (2 a H_ii)
+        const float wF = HFF > 0.f ? __fdividef(0.5f, HFF) * (swap ? a0.y : a1.y) : 0.f;   // 1 / (2 a H_ii), 2 ulp
         const float qFf = (float)qF;
         auto eval = [&](int rS) -> float {
           const float dS = aS * (float)(rS - qS);
@@ -329,6 +316,42 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
           if (!full && phi > lim && phi >= prev) break;
           prev = phi;
         }
+      };
+
+      // ---- test every pair of this thread against the bound ----
+      // A slot in which many lanes of the warp have a pair left is scanned on the spot, with the
+      // pair's data still in registers; otherwise the few pairs wait for the loop below, where a
+      // warp scans only as many rounds as its busiest lane has pairs.
+      unsigned todo = 0;
+#pragma unroll
+      for (int s = 0; s < PPT; ++s) {
+        const unsigned u = (unsigned)tid + (unsigned)NT * s;
+        bool need = false;
+        uint4 e = make_uint4(0u, 0u, 0u, 0u);
+        float g0 = 0.f, g1 = 0.f;
+        if (u < nb) {
+          e = __ldg(trow + u);
+          const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
+          g0 = (float)g_s[m0]; g1 = (float)g_s[m1];
+          const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
+          const float det = fmaf(H00, H11, -h01 * h01);
+          const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
+          const bool full = !(det > 1e-4f * H00 * H11);
+          need = full || !(1.01f * N < -4.f * lim * det);   // 1 % for the rounding of N and det
+        }
+        if (__popc(__ballot_sync(0xFFFFFFFFu, need)) >= 12) {
+          if (need) scan_pair(e, g0, g1);
+        } else if (need) {
+          todo |= 1u << s;
+        }
+      }
+
+      // ---- scan the pairs that are left ----
+      while (todo) {
+        const int s = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const uint4 e = __ldg(trow + (unsigned)tid + (unsigned)NT * s);
+        scan_pair(e, (float)g_s[e.x & 0xFFFFu], (float)g_s[e.x >> 16]);
       }
 
       // ---- team-wide argmin: (change, lowest first coordinate, lowest levels) ----
