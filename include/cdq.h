@@ -93,7 +93,7 @@ typedef struct {
 } cdq_cd_stats;
 
 /*
- * H = X^T X  (paper: Section 3 "Notation"; Algorithm 1 line 2), plus the
+ * H = X^T X  (paper: Section 3 "Notation"; Algorithm 1), plus the
  * optional regulariser of Section 4: H_ii += lambda_rel * mean(diag H).
  *   X          [n, d_in] of type xt, leading dimension ldx (elements, >= d_in).
  *              BF16 input additionally needs X 16-byte aligned and ldx % 8 == 0.

@@ -204,7 +204,7 @@ def bcd_solve(H, W, bits: int, scale, zero, Q, k: int, steps_per_col: int, seed:
 
 
 def gradient(H, W, scale, zero, Q, group_size: int = 0) -> np.ndarray:
-    """G = 2 H (W_hat - W), returned as [d_out, d_in] fp64 (Algorithm 1 line 3, weight units)."""
+    """G = 2 H (W_hat - W), returned as [d_out, d_in] fp64 (the gradient step of Algorithm 1, weight units)."""
     Hf, W, scale, zero, Q = _f32(H), _f64(W), _f32(scale), _f32(zero), _u8(Q)
     d_in, d_out = W.shape
     G = np.empty((d_out, d_in), dtype=np.float64)
@@ -216,7 +216,7 @@ def gradient(H, W, scale, zero, Q, group_size: int = 0) -> np.ndarray:
 
 def cd_solve(H, W, bits: int, scale, zero, Q, steps_per_col: int, group_size: int = 0,
              trace_col: int = -1, want_G: bool = False) -> dict:
-    """Greedy coordinate descent (Algorithm 1 lines 4-8 / Algorithm 4) on every column.
+    """Greedy coordinate descent (the loop of Algorithm 1 / Algorithm 4) on every column.
 
     Returns the new codes (the input Q is not modified) and the statistics."""
     Hf, W, scale, zero = _f32(H), _f64(W), _f32(scale), _f32(zero)

@@ -7,12 +7,12 @@
  * CUDA library shares no code with it and never calls it.
  *
  * What it computes (paper, Section 3):
- *   - H = X^T X                                   (Notation; Algorithm 1 line 2)
+ *   - H = X^T X                                   (Notation; Algorithm 1)
  *   - MinMax / OWC grid and round-to-nearest codes (Eq. 2 and the grid search
  *     over the clipping strength gamma that follows it; per-group form of the
  *     "Initialization" paragraph of the sub-channel section)
- *   - gradient of the layer loss                   (Algorithm 1 line 3)
- *   - greedy coordinate descent                    (Algorithm 1 lines 4-8;
+ *   - gradient of the layer loss                   (Algorithm 1)
+ *   - greedy coordinate descent                    (the loop of Algorithm 1;
  *     Algorithm 4 for sub-channel grids)
  *   - the layer loss  sum_j e_j^T H e_j            (Eq. 1 written with H)
  *   - OWC-CD: greedy descent over per-group clipping strengths (Algorithm 3;
@@ -80,7 +80,7 @@ int cdqo_num_threads(void) {
 }
 
 /* ------------------------------------------------------------------------ */
-/* H = X^T X  (Notation paragraph of Section 3; Algorithm 1 line 2).         */
+/* H = X^T X  (Notation paragraph of Section 3; Algorithm 1).                */
 /* X: [n, d_in] row-major, already widened exactly to fp64.                  */
 /* H64: [d_in, d_in] fp64 result; H32 (may be NULL): the same rounded to     */
 /* fp32, which is what every later stage consumes.                           */
@@ -240,7 +240,7 @@ int cdqo_init_rtn(const double* W, i64 d_in, i64 d_out, const float* H,
 }
 
 /* ------------------------------------------------------------------------ */
-/* Gradient G = 2 H (w_hat - w) for every column (Algorithm 1 line 3 in      */
+/* Gradient G = 2 H (w_hat - w) for every column (Algorithm 1, in             */
 /* weight units).  G: [d_out, d_in] fp64, one column of the layer per row.   */
 /* ------------------------------------------------------------------------ */
 int cdqo_gradient(const float* H, const double* W, i64 d_in, i64 d_out,
@@ -275,7 +275,7 @@ int cdqo_gradient(const float* H, const double* W, i64 d_in, i64 d_out,
 }
 
 /* ------------------------------------------------------------------------ */
-/* Greedy coordinate descent, weight-unit form (Algorithm 1 lines 4-8; the   */
+/* Greedy coordinate descent, weight-unit form (the loop of Algorithm 1; the */
 /* sub-channel Algorithm 4 is the same iteration, see the header).           */
 /* Q is updated in place.  T = passes * d_in steps per column at most.       */
 /* stats_u64[3] = {steps budget (T*d_out), committed moves, columns that ran */
@@ -461,21 +461,22 @@ int cdqo_layer_loss(const float* H, const double* W, i64 d_in, i64 d_out,
 /* State per column: one grid index per group, and G = 2 H e with            */
 /* e = w_hat - w (the vector the algorithm calls v; see the sign note).      */
 /* Table: for every group t and grid point k the residual of that group      */
-/* under Eq. 2 with gamma_k (Algorithm 3 lines 2-6).                         */
+/* under Eq. 2 with gamma_k (the table that Algorithm 3 builds first).       */
 /* Step: for every group t and every k other than its current index, with    */
 /* delta = residual(t, k) - residual(t, current) (a vector over the group),  */
-/*     change(t, k) = delta^T H_tt delta + delta^T G_t        (line 11)      */
-/* take the most negative one, then G <- G + 2 H[:, t] delta  (line 12)      */
-/* and set the group's index to k (line 13).                                 */
+/*     change(t, k) = delta^T H_tt delta + delta^T G_t                       */
+/* take the most negative one, then G <- G + 2 H[:, t] delta                 */
+/* and set the group's index to k.                                           */
 /*                                                                           */
 /* Readings:                                                                 */
 /*  - sign: the paper defines the table entry as w - w_hat and v as          */
 /*    -2 H (w_hat - w) but adds v^T (Delta_old - Delta_new); with those      */
 /*    signs the linear term would be minus the true one.  The change of the  */
 /*    quadratic loss for e -> e + delta is delta^T H delta + 2 e^T H delta,  */
-/*    which is what is computed here, and the update of line 12 is           */
+/*    which is what is computed here, and the algorithm's update of v is     */
 /*    consistent with it;                                                    */
-/*  - start (line 7 says only "initialize"): every group starts at the last  */
+/*  - start (the algorithm does not say from where): every group starts at   */
+/*    the last                                                               */
 /*    grid point (the largest gamma; MinMax when clip_hi = 1);               */
 /*  - ties: lowest group, then lowest grid index; a change is made only if   */
 /*    it strictly lowers the loss, otherwise the column is finished;         */
@@ -512,14 +513,14 @@ int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
 #pragma omp for schedule(dynamic, 1)
     for (i64 j = 0; j < d_out; ++j) {
       for (i64 i = 0; i < d_in; ++i) w[i] = W[i * d_out + j];
-      /* residual table (lines 2-6) */
+      /* residual table */
       for (int k = 0; k < nk; ++k) {
         const double gamma = cdqo_gamma(k, nk, clip_lo, clip_hi);
         for (i64 t = 0; t < ng; ++t)
           grid_rtn_group(w + t * g, g, L, gamma, a + t, b + t, q + t * g);
         residual(w, q, a, b, d_in, g, tab + (size_t)k * d_in);
       }
-      /* start (line 7) and G = 2 H e (lines 8-9) */
+      /* start and G = 2 H e */
       for (i64 t = 0; t < ng; ++t) cur[t] = nk - 1;
       for (i64 i = 0; i < d_in; ++i) e[i] = tab[(size_t)(nk - 1) * d_in + i];
       double loss = quad_form(H, e, d_in, he);
@@ -589,11 +590,13 @@ int cdqo_owc_cd(const double* W, i64 d_in, i64 d_out, const float* H, int bits,
 /* for every block and every assignment r of levels to its coordinates, with */
 /* d_i = a_i (r_i - q_i),                                                    */
 /*     change = sum_i d_i^2 H_ii + 2 sum_{i<m} d_i d_m H_im + sum_i d_i G_i  */
-/* (line 6: (r-q)^T H_bb (r-q) + (r-q)^T g_b in weight units); the most      */
+/* (the algorithm's (r-q)^T H_bb (r-q) + (r-q)^T g_b in weight units); the   */
+/* most                                                                      */
 /* negative change is applied: q_b <- r, G <- G + 2 sum_i d_i H[i, :].       */
 /*                                                                           */
 /* Readings:                                                                 */
-/*  - the partition (line 5 says only "randomly partition"): pi is a         */
+/*  - the partition (the algorithm gives no rule for the random draw): pi is */
+/*    a                                                                      */
 /*    counter-based bijection of {0..d_in-1}, the same on every              */
 /*    implementation: with b = bits of d_in - 1 and mask = 2^b - 1, three    */
 /*    rounds  x <- (x * (2 K_r + 1) + (K_r >> 33)) & mask;  x <- x ^ (x >> s) */

@@ -1,5 +1,5 @@
-// Greedy coordinate descent, batched over all output columns (paper: Algorithm 1 lines
-// 4-8; Algorithm 4 for sub-channel grids; weight-unit form, see include/cdq.h).
+// Greedy coordinate descent, batched over all output columns (paper: the loop of Algorithm 1;
+// Algorithm 4 for sub-channel grids; weight-unit form, see include/cdq.h).
 //
 // One CTA owns one column at a time (columns are handed out through an atomic counter).
 // The column's whole state stays on chip for its T steps: the gradient g (fp64) and the
@@ -7,11 +7,11 @@
 //   1. every thread holds the best move among its coordinates (scored in fp32);
 //   2. warp argmin with two redux.sync, then one shared-memory exchange per CTA;
 //   3. the winning row H[i*, :] is read once, contiguously (H is symmetric, so the
-//      "column i*" of Algorithm 1 line 6 is row i*), 16 bytes per thread per load;
+//      "column i*" in the update of Algorithm 1 is row i*), 16 bytes per thread per load;
 //   4. g += 2 d H[i*, :] in fp64, and each coordinate is re-scored in the same sweep.
 // The best level of a coordinate is the clamped rounding of the vertex of its parabola
 //   r = clamp(rint(q_i - g_i / (2 a_i H_ii)), 0, L),
-// so the level scan of Algorithm 1 line 5 costs O(1) per coordinate.
+// so the scan over the levels in Algorithm 1 costs O(1) per coordinate.
 #include <cstdio>
 #include <cstdlib>
 
@@ -351,7 +351,7 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
 }
 
 // ---------------------------------------------------------------------------
-// Fixed-order fp64 version: the level scan of Algorithm 1 line 5 as written, no fused
+// Fixed-order fp64 version: the scan over the levels of Algorithm 1 as written, no fused
 // multiply-add, ties to the lowest coordinate then the lowest level.  One CTA per column,
 // gradient in global memory.  Small layers only.
 __global__ void __launch_bounds__(128) cd_verify_kernel(CdParams p) {

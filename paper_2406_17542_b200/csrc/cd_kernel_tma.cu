@@ -1,4 +1,4 @@
-// Greedy coordinate descent (paper: Algorithm 1 lines 4-8; Algorithm 4 for sub-channel
+// Greedy coordinate descent (paper: the loop of Algorithm 1; Algorithm 4 for sub-channel
 // grids), the variant for rows of H that have to come from HBM (large d_in) and are 16-byte
 // aligned (d_in % 4 == 0).
 //

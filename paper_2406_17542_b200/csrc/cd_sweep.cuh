@@ -2,8 +2,8 @@
 // the row of H in registers, cd_kernel_tma.cu stages it through shared memory).
 //
 // For a chunk of 4 consecutive coordinates the sweep applies the pending step to the gradient
-// (fp64) and scores the best move of every coordinate (fp32) -- Algorithm 1 lines 5-7 of the
-// paper, with the level scan of line 5 replaced by the clamped rounding of the parabola's vertex
+// (fp64) and scores the best move of every coordinate (fp32) -- the body of the loop of
+// Algorithm 1 of the paper, with its scan over the levels replaced by the clamped rounding of the parabola's vertex
 //   r = clamp(rint(q - g / (2 a H_ii)), 0, L).
 // (Variants that were measured and dropped: a chunk-level running minimum with the winner
 // worked out afterwards, a packed fp64 min carrying score and identity, and an integer-pipe

@@ -1,5 +1,5 @@
 // C = H E in fp64, where E = W_hat - W is the residual of every column.
-// Used for the gradient G = 2 H E (paper: Algorithm 1 line 3, in weight units), for the
+// Used for the gradient G = 2 H E (paper: Algorithm 1, the gradient step, in weight units), for the
 // layer loss sum_j e_j^T H e_j (Eq. 1 written with H) and for the OWC loss of each
 // clipping strength (the objective minimised after Eq. 2).
 //

@@ -1,5 +1,5 @@
 // C = E^T H on the integer tensor cores, exact to a chosen number of bits: the contraction
-// behind the gradient G = 2 H (W_hat - W) (paper: Algorithm 1 line 3), the column losses
+// behind the gradient G = 2 H (W_hat - W) (paper: Algorithm 1, the gradient step), the column losses
 // e_j^T H e_j (paper: Eq. 1 with H = X^T X) and the loss per clipping strength of the OWC
 // search (the minimisation stated after Eq. 2).
 //

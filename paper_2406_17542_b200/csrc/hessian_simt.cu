@@ -1,4 +1,4 @@
-// H = X^T X on the CUDA cores (paper: Section 3 "Notation"; Algorithm 1 line 2).
+// H = X^T X on the CUDA cores (paper: Section 3 "Notation"; Algorithm 1).
 //  - verify kernels: every entry is the ascending-k fp64 sum without fused
 //    multiply-add, rounded once to fp32 (bit-reproducible on a CPU);
 //  - SIMT kernel: tiled, fp64 accumulation, any shape and input type; used for

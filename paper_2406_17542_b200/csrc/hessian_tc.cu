@@ -1,5 +1,5 @@
-// H = X^T X on the 5th-generation tensor cores (paper: Section 3 "Notation"; Algorithm 1
-// line 2).  X is [n, d_in] bf16 row-major, H is [d_in, d_in] fp32.
+// H = X^T X on the 5th-generation tensor cores (paper: Section 3 "Notation"; Algorithm 1).
+// X is [n, d_in] bf16 row-major, H is [d_in, d_in] fp32.
 //
 // The contraction runs over the calibration rows: D[M,N] += A[M,K] B[K,N] with A = X^T,
 // B = X, K = n.  Both operands are slices of the same matrix and are "MN-major" for the

@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
     const long long j = s_col;
     if (j >= p.d_out) break;
 
-    // ---- residual table (Algorithm 3 lines 2-6) and start (line 7) ----
+    // ---- residual table per clipping strength and start (Algorithm 3) ----
     for (long long idx = tid; idx < (long long)nk * d_in; idx += NT) {
       const int k = (int)(idx / d_in);
       const long long i = idx - (long long)k * d_in, t = i / g;
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
     for (long long t = tid; t < ng; t += NT) cur[t] = nk - 1;
     __syncthreads();
 
-    // ---- G = 2 H e and the starting loss (lines 8-9) ----
+    // ---- G = 2 H e and the starting loss ----
     double* G = (!VERIFY && p.Gext) ? p.Gext + j * p.ldg : Gown;
     const double* e0 = R + (size_t)(nk - 1) * d_in;
     double loss = 0.0;
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
     }
     if (tid == 0 && (VERIFY || !p.Gext)) p.col_before[j] = loss;
 
-    // ---- descent over the strengths (lines 10-14) ----
+    // ---- descent over the strengths (the loop of Algorithm 3) ----
     const long long ntask = ng * nk;
     long long nmoves = 0;
     double* quad_s = dyn;
