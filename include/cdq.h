@@ -109,8 +109,8 @@ cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in,
                        size_t ws_bytes, void* stream);
 
 /*
- * The regulariser alone: H_ii += lambda_rel * mean(diag H) (paper: Section 4, "we regularize the
- * Hessian ... by adding lambda I").  For a Hessian that is summed from several parts first (row
+ * The regulariser alone: H_ii += lambda_rel * mean(diag H) (paper: Section 4, the lambda I added to
+ * the Hessian as for GPTQ).  For a Hessian that is summed from several parts first (row
  * chunks, or the row shards of several GPUs after their all-reduce): the parts are formed with
  * lambda_rel = 0 and the sum is regularised once.
  *   H  [d_in, d_in] fp32 device, in/out.  lambda_rel >= 0.
