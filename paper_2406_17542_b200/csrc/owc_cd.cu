@@ -162,18 +162,19 @@ __global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
         __syncthreads();
       }
       // M(k) = H_tt r(t, k): one thread per coordinate i and pass of KC grid points, so that a
-      // value of H feeds KC independent accumulators
+      // value of H feeds KC independent accumulators.  H is symmetric, so M(k)[i] is summed down
+      // column i of the block, H[t0 + q][i]: neighbouring threads read neighbouring addresses.
       const int npass = (nk + KC - 1) / KC;
       for (long long idx = tid; idx < (long long)npass * d_in; idx += NT) {
         const int ps = (int)(idx / d_in);
         const long long i = idx - (long long)ps * d_in, t0 = (i / g) * g;
-        const float* row = p.H + i * d_in + t0;
+        const float* col = p.H + t0 * d_in + i;
         double acc[KC];
 #pragma unroll
         for (int c = 0; c < KC; ++c) acc[c] = 0.0;
 #pragma unroll 4
         for (long long q = 0; q < g; ++q) {
-          const double h = (double)row[q];
+          const double h = (double)col[q * d_in];
 #pragma unroll
           for (int c = 0; c < KC; ++c) {
             const int k = ps * KC + c;
@@ -301,23 +302,30 @@ __global__ void __launch_bounds__(NT, 2) owc_cd_kernel(Params p) {
           G[i] = __dadd_rn(G[i], __dmul_rn(2.0, acc));
         }
       } else {
-        // one thread per row: 4 independent accumulators over the group's g columns (a warp per row
-        // would spend more instructions on the shuffle reduction than on the g / 32 products per lane)
-        for (long long i = tid; i < d_in; i += NT) {
-          const float* row = p.H + i * d_in + ts * g;
-          double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-          long long r = 0;
-          if ((g & 3) == 0 && ((reinterpret_cast<uintptr_t>(row) & 15) == 0)) {
-            for (; r < g; r += 4) {
-              const float4 h = *reinterpret_cast<const float4*>(row + r);
-              a0 = fma((double)h.x, S[r], a0);
-              a1 = fma((double)h.y, S[r + 1], a1);
-              a2 = fma((double)h.z, S[r + 2], a2);
-              a3 = fma((double)h.w, S[r + 3], a3);
+        // G[i] += 2 sum_r H[ts g + r][i] delta_r: H is symmetric, so the g rows of the group are read
+        // along i, four coordinates per thread and 16 bytes per load, as the descent kernels read
+        // their rows; the sum over r runs in ascending order
+        const float* rows = p.H + ts * g * d_in;
+        if ((d_in & 3) == 0 && (reinterpret_cast<uintptr_t>(p.H) & 15) == 0) {
+          for (long long i = 4ll * tid; i < d_in; i += 4ll * NT) {
+            double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 8
+            for (long long r = 0; r < g; ++r) {
+              const float4 h = __ldg(reinterpret_cast<const float4*>(rows + r * d_in + i));
+              const double dl = S[r];
+              a0 = fma((double)h.x, dl, a0);
+              a1 = fma((double)h.y, dl, a1);
+              a2 = fma((double)h.z, dl, a2);
+              a3 = fma((double)h.w, dl, a3);
             }
+            G[i] += 2.0 * a0; G[i + 1] += 2.0 * a1; G[i + 2] += 2.0 * a2; G[i + 3] += 2.0 * a3;
           }
-          for (; r < g; ++r) a0 = fma((double)row[r], S[r], a0);
-          G[i] += 2.0 * ((a0 + a1) + (a2 + a3));
+        } else {
+          for (long long i = tid; i < d_in; i += NT) {
+            double a0 = 0.0;
+            for (long long r = 0; r < g; ++r) a0 = fma((double)rows[r * d_in + i], S[r], a0);
+            G[i] += 2.0 * a0;
+          }
         }
       }
       __syncthreads();
