@@ -51,6 +51,13 @@ def test_workspace_sizes(lib):
     mm = B.workspace_bytes(B.CALL_INIT_RTN, 0, 4096, 4096, B.Grid(2, 128))
     assert owc > mm > 0
     assert B.workspace_bytes(B.CALL_INIT_RTN, 0, 100, 8, B.Grid(2, 7)) == 0   # 100 % 7 != 0
+    # pairs: the table of all steps' pairs (16 bytes per pair and step) on top of the descent's workspace
+    b0 = B.workspace_bytes(B.CALL_BCD_SOLVE, 0, 2048, 16384, g)
+    b256 = B.workspace_bytes(B.CALL_BCD_SOLVE, 256, 2048, 16384, g)
+    assert b0 == cd and b256 - b0 >= 256 * 1024 * 16 and b256 - b0 < 256 * 1024 * 16 + 4096
+    assert B.workspace_bytes(B.CALL_BCD_SOLVE, 256, 2048, 16384, g, "verify") == B.workspace_bytes(B.CALL_CD_SOLVE, 0, 2048, 16384, g, "verify")
+    owc_cd = B.workspace_bytes(B.CALL_INIT_OWC_CD, 0, 4096, 4096, B.Grid(2, 128, 20, 0.5, 1.0))
+    assert owc_cd > 2 * 20 * 4096 * 8
 
 
 def test_bad_arguments_are_rejected_before_any_launch(lib):
@@ -82,6 +89,18 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert st == 2   # ldw < d_out
     st = lib.cdq_cd_solve(dummy, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, -1, 0, None, null, 0, null)
     assert st == 1
+    # pairs: block sizes, odd d_in, too many steps for the table, regulariser arguments
+    bcd = lambda d_in, block, steps: lib.cdq_bcd_solve(dummy, dummy, 0, d_in, 8, 8, ctypes.byref(gd), dummy, dummy, dummy,
+                                                       block, steps, 0, 0, None, null, 0, null)
+    assert bcd(8, 0, 4) == 1
+    assert bcd(9, 2, 4) == 2
+    assert bcd(8, 3, 4) == 2          # 8 % 3 != 0
+    assert bcd(9, 3, 4) == 3          # blocks of three are not built
+    assert bcd(8, 2, 70000) == 3
+    assert bcd(8, 2, 4) == 4          # valid arguments: the workspace is what is missing
+    assert lib.cdq_hessian_add_lambda(null, 8, 0.1, null) == 1
+    assert lib.cdq_hessian_add_lambda(dummy, 0, 0.1, null) == 2
+    assert lib.cdq_hessian_add_lambda(dummy, 8, -1.0, null) == 1
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
