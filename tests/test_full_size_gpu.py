@@ -125,3 +125,9 @@ def test_c1_full_size_pairs_after_the_greedy_descent_sampled_columns():
     per_got = per.cpu().numpy()[cols]
     assert abs(per_got.sum() - ref["loss_after"].sum()) <= LOSS_RTOL * ref["loss_after"].sum()
     assert ref["moves"].sum() > 0
+
+
+def test_c4_shaped_full_d_in_sampled_columns():
+    """The longest columns of the benchmark layers (d_in = 18432, groups of 128, clipping search): the
+    kernel configuration of C4 on 592 of its columns (four per SM), the oracle on four of them."""
+    _run(inputs.CONFIGS["C4"].scaled(d_out=592), rows=8192, n_sample=4)
