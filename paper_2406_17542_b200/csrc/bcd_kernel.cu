@@ -117,7 +117,10 @@ __global__ void bcd2_table_kernel(const float* __restrict__ H, const float* __re
 //      change that some pair reaches (a pair may keep one of its levels);
 //   2. every pair is tested against the bound with the free minimum of its 2 x 2 quadratic,
 //      -N / (4 det), N = g_i^2 H_mm - 2 g_i g_m H_im + g_m^2 H_ii (H is positive
-//      semi-definite, so no assignment of levels does better); most pairs stop here;
+//      semi-definite, so no assignment of levels does better); most pairs stop here.  When the
+//      bound is 0 (no single move lowers the loss: the state the greedy descent leaves) that test
+//      passes every pair, and a sharper one takes its place: a lower bound of the change over
+//      the moves of both coordinates by at least one level each;
 //   3. the pairs that are left are scanned, after the test loop so that a warp scans only as
 //      many rounds as its busiest lane has such pairs: the levels of one coordinate S are
 //      walked outwards from its current level, the level of the other, F, follows in closed
@@ -335,9 +338,26 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
           g0 = (float)g_s[m0]; g1 = (float)g_s[m1];
           const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
           const float det = fmaf(H00, H11, -h01 * h01);
-          const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
           const bool full = !(det > 1e-4f * H00 * H11);
-          need = full || !(1.01f * N < -4.f * lim * det);   // 1 % for the rounding of N and det
+          if (lim == 0.f) {
+            // No single move lowers the loss, so a pair can only win by moving both coordinates.
+            // In level units, with u, v >= 1 the sizes of the two steps, A = a0^2 H00, B = a1^2 H11,
+            // C = a0 a1 H01, rho = |C| / sqrt(A B):
+            //   change >= (1 - rho)(A u^2 + B v^2) - |a0 g0| u - |a1 g1| v     (2 |C| u v <= rho (A u^2 + B v^2))
+            // which splits into one parabola per coordinate; each is bounded below over u >= 1 by its
+            // value at 1 when its vertex is at or left of 1, and by its free minimum otherwise.
+            const float a0 = scale_of(m0).x, a1 = scale_of(m1).x;
+            const float A = a0 * a0 * H00, Bq = a1 * a1 * H11;
+            const float kap = 1.f - fabsf(a0 * a1 * h01) * rsqrtf(A * Bq);
+            const float kA = kap * A, kB = kap * Bq;
+            const float al = fabsf(a0 * g0), be = fabsf(a1 * g1);
+            const float mS = al <= 2.f * kA ? kA - al : -__fdividef(al * al, 4.f * kA);
+            const float mF = be <= 2.f * kB ? kB - be : -__fdividef(be * be, 4.f * kB);
+            need = full || !(mS + mF >= 2e-6f * (A + Bq));   // margin: fp32 rounding of the bound; a NaN (dead coordinate) keeps the pair
+          } else {
+            const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
+            need = full || !(1.01f * N < -4.f * lim * det);   // 1 % for the rounding of N and det
+          }
         }
         if (__popc(__ballot_sync(0xFFFFFFFFu, need)) >= 12) {
           if (need) scan_pair(e, g0, g1);
