@@ -324,22 +324,35 @@ def status_is_workspace(st: int) -> bool:
 
 
 def quantize_layer(X: torch.Tensor, W: torch.Tensor, grid: Grid, passes: int, lambda_rel: float = 0.0, mode="fast",
-                   device="cuda:0", ws: Workspace | None = None, return_host: bool | None = None) -> dict:
+                   device="cuda:0", ws: Workspace | None = None, return_host: bool | None = None,
+                   init: str = "rtn", steps_per_col: int | None = None, bcd_steps: int = 0, seed: int = 0) -> dict:
     """The whole hot path for one layer: Hessian, grid/codes, greedy CD, loss.
 
     X and W may live on the host (pinned memory makes the copies asynchronous): they are then
     copied to `device` first and the codes, scales and zeros are copied back, so that a caller
-    holding host buffers gets host results.  All compute is the four library calls."""
+    holding host buffers gets host results.  All compute is the library's calls.
+
+    The paper's variants around the main loop: init="owc_cd" takes the grid from cdq_init_owc_cd
+    (per-group clipping strengths, needs grid.n_clip > 1) instead of cdq_init_rtn; steps_per_col
+    gives the descent's budget in steps per column instead of passes * d_in; bcd_steps > 0 runs
+    that many steps of block coordinate descent with random pairs from the greedy solution."""
+    if init not in ("rtn", "owc_cd"):
+        raise ValueError("init must be 'rtn' or 'owc_cd'")
     on_host = not X.is_cuda
     if return_host is None:
         return_host = on_host
     Xd = X.to(device, non_blocking=True) if not X.is_cuda else X
     Wd = W.to(device, non_blocking=True) if not W.is_cuda else W
     H = cdq_hessian(Xd, lambda_rel=lambda_rel, mode=mode, ws=ws)
-    scale, zero, Q, gamma = cdq_init_rtn(Wd, grid, H=H if grid.n_clip > 1 else None, mode=mode, ws=ws)
-    stats = cdq_cd_solve(H, Wd, grid, scale, zero, Q, passes, mode=mode, ws=ws)
-    loss = cdq_layer_loss(H, Wd, grid, scale, zero, Q, mode=mode, ws=ws)
-    out = {"H": H, "scale": scale, "zero": zero, "Q": Q, "gamma": gamma, "stats": stats, "loss": loss}
+    if init == "owc_cd":
+        scale, zero, Q, gamma, _ = cdq_init_owc_cd(Wd, grid, H, mode=mode, ws=ws)
+    else:
+        scale, zero, Q, gamma = cdq_init_rtn(Wd, grid, H=H if grid.n_clip > 1 else None, mode=mode, ws=ws)
+    stats = cdq_cd_solve(H, Wd, grid, scale, zero, Q, passes, mode=mode, ws=ws, steps_per_col=steps_per_col)
+    out = {"H": H, "scale": scale, "zero": zero, "Q": Q, "gamma": gamma, "stats": stats}
+    if bcd_steps > 0:
+        out["bcd_stats"] = cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, bcd_steps, seed=seed, mode=mode, ws=ws)
+    out["loss"] = cdq_layer_loss(H, Wd, grid, scale, zero, Q, mode=mode, ws=ws)
     if return_host:
         for k in ("scale", "zero", "Q"):
             out[k] = out[k].to("cpu", non_blocking=False)

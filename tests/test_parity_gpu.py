@@ -207,3 +207,26 @@ def test_regulariser_alone_matches_the_fused_one():
                                atol=1.2e-7 * float(plain.diagonal().max()))
     off = ~torch.eye(cfg.d_in, dtype=torch.bool, device="cuda:0")
     assert torch.equal(parts[off], plain[off])
+
+
+def test_quantize_layer_variants_from_host_buffers():
+    """The one-call path with the paper's variants (OWC-CD grid, reduced budget, pairs after the greedy
+    descent) on pinned host tensors equals the same calls made one by one on device tensors."""
+    cfg = inputs.CONFIGS["C2"].scaled(d_in=512, d_out=160, n=2048, seed=19)
+    X, W = inputs.make_layer(cfg)
+    grid = grid_of(cfg)
+    out = B.quantize_layer(X.pin_memory(), W.pin_memory(), grid, cfg.passes, init="owc_cd", steps_per_col=cfg.d_in // 2,
+                           bcd_steps=64, seed=5)
+    assert not out["Q"].is_cuda and not out["scale"].is_cuda
+    Xd, Wd = X.to("cuda:0"), W.to("cuda:0")
+    H = B.cdq_hessian(Xd)
+    scale, zero, Q, gamma, _ = B.cdq_init_owc_cd(Wd, grid, H)
+    B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, steps_per_col=cfg.d_in // 2)
+    l_cd = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q)
+    st = B.cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, 64, seed=5)
+    loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q)
+    assert torch.equal(out["Q"], Q.cpu()) and torch.equal(out["scale"], scale.cpu())
+    assert out["loss"] == loss and out["bcd_stats"]["committed"] == st["committed"]
+    assert loss <= l_cd
+    with pytest.raises(ValueError):
+        B.quantize_layer(Xd, Wd, grid, 1, init="gptq")
