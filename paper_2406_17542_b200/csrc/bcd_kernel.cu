@@ -322,23 +322,30 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
       };
 
       // ---- test every pair of this thread against the bound ----
-      // A slot in which many lanes of the warp have a pair left is scanned on the spot, with the
-      // pair's data still in registers; otherwise the few pairs wait for the loop below, where a
-      // warp scans only as many rounds as its busiest lane has pairs.
+      // The table entries of up to 8 pairs are requested together, so that a step waits for the
+      // table once or twice, not once per pair; the pairs that are left wait for the loop below,
+      // where a warp scans only as many rounds as its busiest lane has pairs.
       unsigned todo = 0;
+      constexpr int TB = PPT < 8 ? PPT : 8;
 #pragma unroll
-      for (int s = 0; s < PPT; ++s) {
-        const unsigned u = (unsigned)tid + (unsigned)NT * s;
-        bool need = false;
-        uint4 e = make_uint4(0u, 0u, 0u, 0u);
-        float g0 = 0.f, g1 = 0.f;
-        if (u < nb) {
-          e = __ldg(trow + u);
+      for (int s0 = 0; s0 < PPT; s0 += TB) {
+        uint4 ev[TB];
+#pragma unroll
+        for (int k = 0; k < TB; ++k) {
+          const unsigned u = (unsigned)tid + (unsigned)NT * (s0 + k);
+          ev[k] = u < nb ? __ldg(trow + u) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < TB; ++k) {
+          const unsigned u = (unsigned)tid + (unsigned)NT * (s0 + k);
+          if (u >= nb) continue;
+          const uint4 e = ev[k];
           const unsigned m0 = e.x & 0xFFFFu, m1 = e.x >> 16;
-          g0 = (float)g_s[m0]; g1 = (float)g_s[m1];
+          const float g0 = (float)g_s[m0], g1 = (float)g_s[m1];
           const float H00 = __uint_as_float(e.z), H11 = __uint_as_float(e.w), h01 = __uint_as_float(e.y);
           const float det = fmaf(H00, H11, -h01 * h01);
           const bool full = !(det > 1e-4f * H00 * H11);
+          bool need;
           if (lim == 0.f) {
             // No single move lowers the loss, so a pair can only win by moving both coordinates.
             // In level units, with u, v >= 1 the sizes of the two steps, A = a0^2 H00, B = a1^2 H11,
@@ -358,11 +365,7 @@ bcd2_kernel(CdParams p, const uint4* __restrict__ tab, int g_in_smem, int a_in_s
             const float N = fmaf(g1 * g1, H00, fmaf(g0 * g0, H11, -2.f * g0 * g1 * h01));
             need = full || !(1.01f * N < -4.f * lim * det);   // 1 % for the rounding of N and det
           }
-        }
-        if (__popc(__ballot_sync(0xFFFFFFFFu, need)) >= 12) {
-          if (need) scan_pair(e, g0, g1);
-        } else if (need) {
-          todo |= 1u << s;
+          if (need) todo |= 1u << (s0 + k);
         }
       }
 
