@@ -595,6 +595,7 @@ cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char*
   if (nb <= 2048) return launch_bcd_cfg<4, 512, 2>(p, tab, team(4), st);
   if (nb <= 7168) return launch_bcd_cfg<8, 896, 1>(p, tab, team(8), st);
   if (nb <= 8192) return launch_bcd_cfg<8, 1024, 1>(p, tab, team(8), st);
+  if (nb <= 9216) return launch_bcd_cfg<12, 768, 1>(p, tab, team(12), st);
   return launch_bcd_cfg<16, 1024, 1>(p, tab, team(16), st);
 }
 

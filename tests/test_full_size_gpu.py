@@ -131,3 +131,35 @@ def test_c4_shaped_full_d_in_sampled_columns():
     """The longest columns of the benchmark layers (d_in = 18432, groups of 128, clipping search): the
     kernel configuration of C4 on 592 of its columns (four per SM), the oracle on four of them."""
     _run(inputs.CONFIGS["C4"].scaled(d_out=592), rows=8192, n_sample=4)
+
+
+def test_c4_shaped_pairs_after_the_greedy_descent_sampled_columns():
+    """Pairs on the longest columns (d_in = 18432, groups of 128: the 12-pairs-per-thread configuration),
+    from the greedy solution, on 148 columns; the oracle takes the same stages on three of them."""
+    cfg = inputs.CONFIGS["C4"].scaled(d_out=148, n_clip=1, clip_lo=1.0, clip_hi=1.0)
+    dev = "cuda:0"
+    Hd = _h_from_rows(cfg, 8192)
+    Wd = inputs.make_w(cfg, device=dev)
+    g = grid_of(cfg)
+    T, seed = 64, 8
+    scale, zero, Q, _ = B.cdq_init_rtn(Wd, g)
+    B.cdq_cd_solve(Hd, Wd, g, scale, zero, Q, cfg.passes)
+    stats = B.cdq_bcd_solve(Hd, Wd, g, scale, zero, Q, 2, T, seed=seed)
+    loss, per = B.cdq_layer_loss(Hd, Wd, g, scale, zero, Q, per_col=True)
+    assert B.load().cdq_last_device_status() == 0
+    assert stats["steps"] == T * cfg.d_out and stats["loss_after"] <= stats["loss_before"]
+    np.testing.assert_allclose(stats["loss_after"], loss, rtol=1e-5)
+
+    cols = np.array([5, 71, 140])
+    H32 = Hd.cpu().numpy()
+    Wc = Wd[:, torch.from_numpy(cols).to(dev)].cpu()
+    init = oracle.init_rtn(Wc, cfg.bits, cfg.group_size, 1, 1.0, 1.0)
+    cd = oracle.cd_solve(H32, Wc, cfg.bits, init["scale"], init["zero"], init["Q"], cfg.passes * cfg.d_in, cfg.group_size)
+    ref = oracle.bcd_solve(H32, Wc, cfg.bits, init["scale"], init["zero"], cd["Q"], 2, T, seed=seed,
+                           group_size=cfg.group_size)
+    got = Q.cpu().numpy()[:, cols]
+    agree = float((got == ref["Q"]).mean())
+    forked = int((got != ref["Q"]).any(axis=0).sum())
+    assert agree >= CODE_AGREE or (forked <= 1 and agree >= 0.99), (agree, forked)
+    per_got = per.cpu().numpy()[cols]
+    assert abs(per_got.sum() - ref["loss_after"].sum()) <= LOSS_RTOL * ref["loss_after"].sum()
