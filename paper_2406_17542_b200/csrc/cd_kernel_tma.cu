@@ -4,7 +4,8 @@
 //
 // Same step as cd_kernel.cu -- score, argmin, read row i*, update the gradient -- but the row
 // H[i*, :] is fetched by bulk asynchronous copies (cp.async.bulk, no multicast) into shared
-// memory, one copy and one mbarrier per chunk slot of the team, issued by a single thread.
+// memory, one copy and one mbarrier per chunk slot of the team (or one for the whole row, see PS),
+// each issued by a single thread.
 // The copy engine keeps the whole row in flight at once (loads issued by the threads themselves
 // did not: the SM tracks only so many outstanding misses), the sweep starts on the first piece
 // while the others are still landing, and the row no longer occupies 32 registers per thread.
@@ -52,12 +53,16 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-
 // NCH chunk slots per thread; the team covers ceil(d_in / 4) <= NT * NCH chunks.
 template <int NCH, int MAXNT, int MINB, int SMODE>
 __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
-  __shared__ __align__(8) unsigned long long s_bar[NCH];
+  // chunk slots per bulk copy: the 896 x 4 team (rows of up to 57 KB) is quickest with the whole row in one
+  // copy (322 ms against 333 with two and 350 with four on a C3-shaped layer), the 768 x 6 team (74 KB rows,
+  // 24 coordinates per thread) with one copy per slot (616 ms against 626 with three and 651 with two)
+  constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : 1;
+  constexpr int NP = NCH / PS;                              // bulk copies per row
+  __shared__ __align__(8) unsigned long long s_bar[NP];
   __shared__ __align__(8) uint2 s_exch[2][32];
   __shared__ int s_col;
 
@@ -87,12 +92,12 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   for (int t = tid; t < NCH * NT; t += NT) row_s[t] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid == 0) {
 #pragma unroll
-    for (int k = 0; k < NCH; ++k) mbar_init(smem_u32(&s_bar[k]), 1);
+    for (int k = 0; k < NP; ++k) mbar_init(smem_u32(&s_bar[k]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // bytes of the row piece behind chunk slot k (0 when the slot lies past the row)
   auto piece_bytes = [&](int k) -> uint32_t {
-    const int lo = NT * k, hi = min(NT * (k + 1), nchs);
+    const int lo = NT * PS * k, hi = min(NT * PS * (k + 1), nchs);
     return hi > lo ? (uint32_t)(hi - lo) * 16u : 0u;
   };
   __syncthreads();
@@ -159,13 +164,13 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       {
         const float* src = p.H + rowoff;
 #pragma unroll
-        for (int k = 0; k < NCH; ++k) {
-          const bool issuer = nwarps >= NCH ? (warp == k && lane == 0) : tid == 0;
+        for (int k = 0; k < NP; ++k) {
+          const bool issuer = nwarps >= NP ? (warp == k && lane == 0) : tid == 0;
           const uint32_t bytes = piece_bytes(k);
           if (issuer && bytes) {
             const uint32_t bar = smem_u32(&s_bar[k]);
             mbar_expect_tx(bar, bytes);
-            bulk_load(smem_u32(row_s + (size_t)NT * k), src + (size_t)NT * k * 4, bytes, bar);
+            bulk_load(smem_u32(row_s + (size_t)NT * PS * k), src + (size_t)NT * PS * k * 4, bytes, bar);
           }
         }
       }
@@ -178,8 +183,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         const float4 hs = __ldg(reinterpret_cast<const float4*>(p.hs) + cs);
         float a, ia;
         chunk_scale(k, a, ia);
-        if (exact || NT * k < nchs) {
-          if (!mbar_wait(smem_u32(&s_bar[k]), phase)) timed_out = true;
+        if ((k % PS) == 0 && (exact || NT * k < nchs)) {
+          if (!mbar_wait(smem_u32(&s_bar[k / PS]), phase)) timed_out = true;
         }
         const float4 rv = row_s[cs];
         double gk[4] = {g[4 * k], g[4 * k + 1], g[4 * k + 2], g[4 * k + 3]};
