@@ -163,3 +163,9 @@ def test_c4_shaped_pairs_after_the_greedy_descent_sampled_columns():
     assert agree >= CODE_AGREE or (forked <= 1 and agree >= 0.99), (agree, forked)
     per_got = per.cpu().numpy()[cols]
     assert abs(per_got.sum() - ref["loss_after"].sum()) <= LOSS_RTOL * ref["loss_after"].sum()
+
+
+def test_mid_size_columns_sampled():
+    """Columns between the L2-served and the longest ones (d_in = 6144: two 256-thread teams per SM, rows by one
+    bulk copy each), 296 columns, the oracle on six of them."""
+    _run(inputs.CONFIGS["C3"].scaled(d_in=6144, d_out=296, seed=61), rows=8192, n_sample=6)
