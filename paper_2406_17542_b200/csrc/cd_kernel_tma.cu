@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
   // chunk slots per bulk copy: the 896 x 4 team (rows of up to 57 KB) is quickest with the whole row in one
   // copy (322 ms against 333 with two and 350 with four on a C3-shaped layer), the 768 x 6 team (74 KB rows,
-  // 24 coordinates per thread) with one copy per slot (616 ms against 626 with three, 651 with two and 731 with one);
+  // 24 coordinates per thread) with one copy per slot (616 ms against 640 with twelve, 626 with three, 651 with two and 731 with one);
   // the 256 x 8 teams of the columns in between, two per SM, again with one copy for the row (d_in = 8192:
   // 105 ms against 137 with eight copies)
   constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : ((NCH == 8 && MAXNT == 256) ? 8 : 1);
