@@ -169,3 +169,9 @@ def test_mid_size_columns_sampled():
     """Columns between the L2-served and the longest ones (d_in = 6144: two 256-thread teams per SM, rows by one
     bulk copy each), 296 columns, the oracle on six of them."""
     _run(inputs.CONFIGS["C3"].scaled(d_in=6144, d_out=296, seed=61), rows=8192, n_sample=6)
+
+
+def test_ragged_long_columns_sampled():
+    """d_in = 11008 (not a multiple of the team's footprint: the last chunk slots reach past the row), rows
+    from HBM by one bulk copy, 296 columns, the oracle on four of them."""
+    _run(inputs.CONFIGS["C3"].scaled(d_in=11008, d_out=296, seed=67), rows=8192, n_sample=4)
