@@ -337,7 +337,8 @@ def main():
                     "executed_frac_of_bf16_sustained_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                     "executed_frac_of_bf16_burst_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                     "note": "symmetric rank-k update: only lower-triangle tiles are computed; the fraction counts executed flops only"},
-        "roofline": {"kernel": "bcd2_kernel" if args.block == 2 else "cd_fast_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        "roofline": {"kernel": "bcd2_kernel" if args.block == 2 else ("cd_tma_kernel" if cfg.d_in > 2048 and cfg.d_in % 4 == 0
+                                                                  else "cd_fast_kernel"), "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.block == 1 else None, "algorithmic_bytes": alg_bytes,

@@ -61,8 +61,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   // copy (322 ms against 333 with two and 350 with four on a C3-shaped layer), the 768 x 6 team (74 KB rows,
   // 24 coordinates per thread) with one copy per slot (616 ms against 640 with twelve, 626 with three, 651 with two and 731 with one);
   // the 256 x 8 teams of the columns in between, two per SM, again with one copy for the row (d_in = 8192:
-  // 105 ms against 137 with eight copies)
-  constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : ((NCH == 8 && MAXNT == 256) ? 8 : 1);
+  // 105 ms against 137 with eight copies), and so the 256 x 4 teams of d_in <= 4096
+  constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : ((NCH == 8 && MAXNT == 256) ? 8 : ((NCH == 4 && MAXNT == 256) ? 4 : 1));
   constexpr int NP = NCH / PS;                              // bulk copies per row
   __shared__ __align__(8) unsigned long long s_bar[NP];
   __shared__ __align__(8) uint2 s_exch[2][32];
