@@ -113,7 +113,9 @@ cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in,
  * the Hessian as for GPTQ).  For a Hessian that is summed from several parts first (row
  * chunks, or the row shards of several GPUs after their all-reduce): the parts are formed with
  * lambda_rel = 0 and the sum is regularised once.
- *   H  [d_in, d_in] fp32 device, in/out.  lambda_rel >= 0.
+ *   H  [d_in, d_in] fp32 device, in/out, owned by the caller.  lambda_rel >= 0 (0: nothing is launched).
+ * Errors: CDQ_ERR_INVALID_ARG (NULL H, negative or NaN lambda_rel), CDQ_ERR_SHAPE (d_in < 1),
+ * CDQ_ERR_UNSUPPORTED (d_in > 65535), CDQ_ERR_CUDA.  No workspace; asynchronous on `stream`.
  */
 cdq_status cdq_hessian_add_lambda(float* H, long long d_in, float lambda_rel, void* stream);
 
