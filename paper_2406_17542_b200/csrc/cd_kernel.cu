@@ -329,17 +329,16 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
   p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
-  // CDQ_CD_KERNEL=plain in the environment keeps the rows in registers (no bulk copies);
-  // CDQ_CD_KERNEL=tma stages them through shared memory whenever the shape allows
-  static const int force = [] {
-    const char* e = getenv("CDQ_CD_KERNEL");
-    return !e ? 0 : (e[0] == 'p' ? 1 : (e[0] == 't' ? 2 : 0));
-  }();
   const long long d = ly.d_in;
+  if (steps_per_col <= 0) return cudaSuccess;   // nothing to do: the counters stay zero, the codes untouched
+  // rows that stream from HBM: two columns in flight per SM
+  if (d > 4096) {
+    const cudaError_t e = launch_cd_pair(p, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
   // short rows (up to 8 KB) are quickest as plain loads into registers; longer ones as bulk copies into
-  // shared memory (one copy per row where the team is small: C2-shaped 62.5 -> 60.2 ms, C1-shaped 48.2 -> 47.7)
-  const bool want_tma = force == 2 || (force == 0 && d > 2048);
-  if (want_tma) {
+  // shared memory
+  if (d > 2048) {
     const cudaError_t e = launch_cd_tma(p, st);
     if (e != cudaErrorNotSupported) return e;
   }
