@@ -38,6 +38,12 @@
  *     that codes can be compared bit for bit with a CPU implementation of the same steps; it is
  *     meant for small layers.
  *   - H must be finite; the descent multiplies rows of H by a zero step in its first sweep.
+ *   - H must be 16-byte aligned wherever it is passed (it is read with 16-byte vector loads and
+ *     bulk copies); a misaligned H is CDQ_ERR_INVALID_ARG before anything is launched.
+ *   - Environment (read once per process, for debugging only): CDQ_DEBUG_SYNC=1 synchronises the
+ *     device after every step of a call, so that an asynchronous kernel failure is attributed to
+ *     the step that caused it; CDQ_BCD_G=global keeps the gradient of cdq_bcd_solve in global
+ *     memory at every size (the path that only layers of more than ~25 K inputs take otherwise).
  */
 #ifndef CDQ_H_
 #define CDQ_H_
@@ -282,8 +288,27 @@ cdq_status cdq_layer_loss_static(const float* H, const void* W, cdq_dtype wt, lo
 size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long long d_out,
                            const cdq_grid_desc* grid, cdq_mode mode);
 
-/* Reads and clears the device-side status word (synchronises the device). */
+/* Reads and clears the device-side status word (synchronises the device): CDQ_OK,
+ * CDQ_ERR_TIMEOUT (a bounded wait on a copy barrier ran out) or CDQ_ERR_CUDA (a kernel stopped on
+ * an internal consistency check; cdq_last_error_detail() names it). */
 cdq_status cdq_last_device_status(void);
+
+/* Kernels this library has launched in this process so far (all entry points, all streams).
+ * Host-side count, no synchronisation.  (No counterpart in the paper: bookkeeping for benchmarks.) */
+unsigned long long cdq_kernel_launches(void);
+
+/*
+ * Diagnostics for the failure path (no counterpart in the paper).  Neither faults nor hangs the GPU.
+ * cdq_debug_expire_wait: launches one small CTA on `stream` that arms a copy barrier for bytes that
+ *   nothing will ever send and waits on it with the library's bounded wait (limit_cycles clock
+ *   cycles, 1 .. 2^31); the wait runs out, the kernel records that in the device status word
+ *   and returns.  The next cdq_last_device_status() (or synchronising call) reports CDQ_ERR_TIMEOUT.
+ * cdq_debug_set_device_status: writes `flag` (0 ok, 1 wait ran out, 2 consistency check) into the
+ *   status word from the host, synchronously.
+ * Errors: CDQ_ERR_INVALID_ARG (limit or flag out of range), CDQ_ERR_CUDA.
+ */
+cdq_status cdq_debug_expire_wait(long long limit_cycles, void* stream);
+cdq_status cdq_debug_set_device_status(int flag);
 
 /* Text of the most recent CDQ_ERR_CUDA in this process (CUDA error name, the failing step),
  * or of a size rejection by cdq_layer_loss_static; an empty string if there was none.  The pointer stays valid; the text is overwritten by

@@ -26,7 +26,8 @@ _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, M
 
 EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
-           "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version"]
+           "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version",
+           "cdq_kernel_launches", "cdq_debug_expire_wait", "cdq_debug_set_device_status"]
 
 
 class CdqError(RuntimeError):
@@ -77,6 +78,11 @@ def load():
     lib.cdq_status_string.restype = ctypes.c_char_p
     lib.cdq_status_string.argtypes = [ci]
     lib.cdq_last_device_status.restype = ci
+    lib.cdq_kernel_launches.restype = ctypes.c_ulonglong
+    lib.cdq_debug_expire_wait.restype = ci
+    lib.cdq_debug_expire_wait.argtypes = [ll, vp]
+    lib.cdq_debug_set_device_status.restype = ci
+    lib.cdq_debug_set_device_status.argtypes = [ci]
     lib.cdq_last_error_detail.restype = ctypes.c_char_p
     lib.cdq_workspace_bytes.restype = sz
     lib.cdq_workspace_bytes.argtypes = [ci, ll, ll, ll, gp, ci]

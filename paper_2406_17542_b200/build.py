@@ -16,7 +16,7 @@ INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libcdq.so")
 
-SOURCES = ["api.cu", "hessian_simt.cu", "hessian_tc.cu", "init_rtn.cu", "owc_cd.cu", "gemm_f64.cu", "gemm_i8.cu", "cd_kernel.cu", "cd_kernel_tma.cu", "cd_kernel_pair.cu", "bcd_kernel.cu",
+SOURCES = ["api.cu", "hessian_simt.cu", "hessian_tc.cu", "init_rtn.cu", "owc_cd.cu", "gemm_f64.cu", "gemm_i8.cu", "cd_kernel.cu", "cd_kernel_tma.cu", "bcd_kernel.cu",
            "layer_loss_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--fmad=true"]

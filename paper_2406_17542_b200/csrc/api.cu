@@ -4,9 +4,26 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
+#include "async_copy.cuh"
 #include "common.cuh"
 
 namespace cdq {
+
+// One CTA: a copy barrier armed for bytes that never come, waited on with the bounded wait.
+__global__ void expire_wait_kernel(long long limit_cycles, int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+    mbar_expect_tx(smem_u32(&bar), 16);
+  }
+  __syncthreads();
+  if (!mbar_wait_cycles(smem_u32(&bar), 0, limit_cycles) && threadIdx.x == 0)
+    atomicCAS(status, (int)kFlagOk, (int)kFlagWaitTimeout);
+}
 
 __device__ int g_device_status = 0;
 
@@ -15,6 +32,9 @@ int* device_status_word() {
   if (cudaGetSymbolAddress((void**)&p, g_device_status) != cudaSuccess) return nullptr;
   return p;
 }
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 static char g_error_detail[256] = "";
 void set_error_detail(const char* text) { snprintf(g_error_detail, sizeof(g_error_detail), "%s", text); }
@@ -71,7 +91,7 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   w.ldg = (d_in + 3) / 4 * 4;
   w.d_pad = cd_fast_pad(d_in);
-  w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+  w.tc = mode == CDQ_MODE_FAST && gemm_tc_supported(d_in, d_out);
   // the loss of a descended solution is a sum with heavy cancellation (the descent tunes e against the
   // large entries of H): it takes the same slice depth as the gradient; the shallower setting serves
   // the OWC search, whose residuals are plain rounding errors
@@ -109,12 +129,6 @@ void note_cuda_error(cudaError_t e, const char* what, int line) {
 
 // CDQ_DEBUG_SYNC=1 in the environment synchronises the device after every step, so that an
 // asynchronous kernel failure is attributed to the step that caused it.
-}  // namespace
-bool gemm_tc_enabled() {
-  static const bool on = [] { const char* e = getenv("CDQ_GEMM"); return !(e && e[0] == 's'); }();
-  return on;
-}
-namespace {
 
 bool debug_sync() {
   static int v = -1;
@@ -134,6 +148,25 @@ bool debug_sync() {
       return CDQ_ERR_CUDA;                              \
     }                                                   \
   } while (0)
+
+// Two events per device, made on first use and kept: cdq_cd_solve times its descent kernel with them.
+cudaError_t timing_events(cudaEvent_t* ev0, cudaEvent_t* ev1) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static cudaEvent_t evs[kMaxDevices][2] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < 2; ++i)
+    if (!evs[dev][i]) {
+      e = cudaEventCreate(&evs[dev][i]);
+      if (e != cudaSuccess) { evs[dev][i] = nullptr; return e; }
+    }
+  *ev0 = evs[dev][0]; *ev1 = evs[dev][1];
+  return cudaSuccess;
+}
 
 cdq_status read_device_status_after_sync() {
   int flag = 0;
@@ -155,7 +188,9 @@ using namespace cdq;
 
 extern "C" {
 
-int cdq_version(void) { return 100; }
+int cdq_version(void) { return 200; }
+
+unsigned long long cdq_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* cdq_status_string(cdq_status s) {
   switch (s) {
@@ -175,6 +210,22 @@ const char* cdq_last_error_detail(void) { return g_error_detail; }
 cdq_status cdq_last_device_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return CDQ_ERR_CUDA;
   return read_device_status_after_sync();
+}
+
+cdq_status cdq_debug_expire_wait(long long limit_cycles, void* stream) {
+  if (limit_cycles < 1 || limit_cycles > (1ll << 31)) return CDQ_ERR_INVALID_ARG;
+  int* status = device_status_word();
+  if (!status) return CDQ_ERR_CUDA;
+  { expire_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_cycles, status); count_launch(); }
+  CDQ_CUDA(cudaGetLastError());
+  return CDQ_OK;
+}
+
+cdq_status cdq_debug_set_device_status(int flag) {
+  if (flag < (int)kFlagOk || flag > (int)kFlagBadIndex) return CDQ_ERR_INVALID_ARG;
+  CDQ_CUDA(cudaDeviceSynchronize());
+  CDQ_CUDA(cudaMemcpyToSymbol(g_device_status, &flag, sizeof(int)));
+  return CDQ_OK;
 }
 
 size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long long d_out, const cdq_grid_desc* grid,
@@ -212,6 +263,7 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
 cdq_status cdq_hessian(const void* X, cdq_dtype xt, long long n, long long d_in, long long ldx, float lambda_rel,
                        int accumulate, float* H, cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {
   if (!X || !H || !valid_dtype(xt) || !valid_mode(mode) || !(lambda_rel >= 0.f)) return CDQ_ERR_INVALID_ARG;
+  if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
   if (n < 1 || d_in < 1 || ldx < d_in) return CDQ_ERR_SHAPE;
   if (d_in > 65535) return CDQ_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
@@ -249,7 +301,7 @@ cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);
   if (s != CDQ_OK) return s;
-  if (grid->n_clip > 1 && !H) return CDQ_ERR_INVALID_ARG;
+  if (grid->n_clip > 1 && (!H || !aligned16(H))) return CDQ_ERR_INVALID_ARG;
   Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, nullptr, nullptr);
   if (ly.ng > 65535) return CDQ_ERR_UNSUPPORTED;
   s = check_ws(ws, ws_bytes, init_rtn_workspace(d_in, d_out, ly.g, grid->n_clip, mode));
@@ -263,6 +315,7 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
                            float* gamma_out, cdq_owc_cd_stats* stats, cdq_mode mode, void* ws, size_t ws_bytes,
                            void* stream) {
   if (!W || !H || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode)) return CDQ_ERR_INVALID_ARG;
+  if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
   cdq_status s = check_layer_shape(d_in, d_out, ldw);
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);
@@ -287,6 +340,7 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
                                 cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
   if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || steps_per_col < 0)
     return CDQ_ERR_INVALID_ARG;
+  if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
   if (block < 1) return CDQ_ERR_INVALID_ARG;
   if (block > 1 && d_in % block) return CDQ_ERR_SHAPE;
   if (block > 1 && !bcd_supported(d_in, block)) return CDQ_ERR_UNSUPPORTED;
@@ -326,10 +380,7 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   CDQ_CUDA(launch_transpose_u8(Q, d_in, d_out, d_out, Qt, L.ldg, st));
   CDQ_CUDA(cudaMemsetAsync(ctr, 0, sizeof(CdCounters), st));
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  if (stats) {
-    CDQ_CUDA(cudaEventCreate(&ev0));
-    CDQ_CUDA(cudaEventCreate(&ev1));
-  }
+  if (stats) CDQ_CUDA(timing_events(&ev0, &ev1));
   // shapes the fast kernels do not cover (a group size that is not a multiple of 4, very long
   // columns) take the fixed-order fp64 kernel: slower, same result
   const bool fast_cd = mode == CDQ_MODE_FAST && cd_fast_supported(d_in, ly.g);
@@ -363,8 +414,6 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
     float ms = 0.f;
     CDQ_CUDA(cudaEventElapsedTime(&ms, ev0, ev1));
     stats->kernel_ms = (double)ms;
-    cudaEventDestroy(ev0);
-    cudaEventDestroy(ev1);
     return read_device_status_after_sync();
   }
   return CDQ_OK;
@@ -398,6 +447,7 @@ cdq_status cdq_layer_loss(const float* H, const void* W, cdq_dtype wt, long long
                           const cdq_grid_desc* grid, const float* scale, const float* zero, const unsigned char* Q,
                           double* loss, double* per_col, cdq_mode mode, void* ws, size_t ws_bytes, void* stream) {
   if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode)) return CDQ_ERR_INVALID_ARG;
+  if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
   cdq_status s = check_layer_shape(d_in, d_out, ldw);
   if (s != CDQ_OK) return s;
   s = check_grid(grid, d_in);

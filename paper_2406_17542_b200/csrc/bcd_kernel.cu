@@ -560,7 +560,7 @@ static cudaError_t launch_bcd_cfg(const CdParams& p, const uint4* tab, int nt, c
   if (per_sm < 1) return cudaErrorInvalidConfiguration;
   long long blocks = (long long)sms * per_sm;
   if (blocks > p.d_out) blocks = p.d_out;
-  kern<<<(unsigned)blocks, nt, smem, st>>>(p, tab, g_in_smem, a_in_smem);
+  { kern<<<(unsigned)blocks, nt, smem, st>>>(p, tab, g_in_smem, a_in_smem); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -578,7 +578,7 @@ cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char*
   if (!p.status) return cudaErrorInvalidSymbol;
   p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
   if (!fast) {
-    bcd2_verify_kernel<<<(unsigned)ly.d_out, 128, 0, st>>>(p, seed, bcd_shape(ly.d_in));
+    { bcd2_verify_kernel<<<(unsigned)ly.d_out, 128, 0, st>>>(p, seed, bcd_shape(ly.d_in)); count_launch(); }
     return cudaGetLastError();
   }
   const long long nb = ly.d_in / 2;
@@ -586,7 +586,7 @@ cudaError_t launch_bcd(const Layer& ly, double* G, long long ldg, unsigned char*
   if (steps_per_col > 0) {
     if (steps_per_col > 65535) return cudaErrorNotSupported;  // steps index a grid dimension
     dim3 grid((unsigned)((nb + 255) / 256), (unsigned)steps_per_col);
-    bcd2_table_kernel<<<grid, 256, 0, st>>>(ly.H, hdiag, (unsigned)ly.d_in, seed, bcd_shape(ly.d_in), tab);
+    { bcd2_table_kernel<<<grid, 256, 0, st>>>(ly.H, hdiag, (unsigned)ly.d_in, seed, bcd_shape(ly.d_in), tab); count_launch(); }
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -12,9 +12,6 @@
 // The best level of a coordinate is the clamped rounding of the vertex of its parabola
 //   r = clamp(rint(q_i - g_i / (2 a_i H_ii)), 0, L),
 // so the scan over the levels in Algorithm 1 costs O(1) per coordinate.
-#include <cstdio>
-#include <cstdlib>
-
 #include "common.cuh"
 #include "cd_params.cuh"
 #include "cd_sweep.cuh"
@@ -40,7 +37,7 @@ __global__ void diag_kernel(const float* __restrict__ H, long long d_in, long lo
 }
 
 cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* hs, cudaStream_t st) {
-  diag_kernel<<<(unsigned)((d_pad + 255) / 256), 256, 0, st>>>(H, d_in, d_pad, hdiag, hs);
+  { diag_kernel<<<(unsigned)((d_pad + 255) / 256), 256, 0, st>>>(H, d_in, d_pad, hdiag, hs); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -63,7 +60,7 @@ __global__ void transpose_u8_kernel(const unsigned char* __restrict__ src, long 
 cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long long cols, long long ld_src,
                                 unsigned char* dst, long long ld_dst, cudaStream_t st) {
   dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32)), block(32, 8);
-  transpose_u8_kernel<<<grid, block, 0, st>>>(src, rows, cols, ld_src, dst, ld_dst);
+  { transpose_u8_kernel<<<grid, block, 0, st>>>(src, rows, cols, ld_src, dst, ld_dst); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -164,7 +161,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
     }
 
     // ---- descent ----
-    // The first sweep only scores: it "applies" a step of size zero along row 0.
+    // The first sweep only scores: it "applies" a step of size zero along row 0.  (T >= 1: the launcher
+    // skips the kernel for an empty budget.)
     long long step = 0;
     const float* rp = p.H;
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
@@ -203,7 +201,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
         sweep_chunk<SMODE>(gk, row[k], hd, hs, qp[k], c2, a, ia, top, k, sb);
         g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
       }
-      if (step >= p.T) break;
 
       // ---- team-wide argmin: (decrease, lowest coordinate, lowest level) ----
       unsigned key, packed;
@@ -239,7 +236,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
       c2 = 2.0 * ((double)astar * (double)dri);
       rp = p.H + (long long)istar * d_in;
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
-      ++step;
+      // budget used up: the gradient after the last move is never read, so no sweep follows it
+      if (++step >= p.T) break;
     }
     if (tid == 0) {
       if (done) ++my_converged;
@@ -289,7 +287,7 @@ static cudaError_t launch_cd_cfg(CdParams p, int nt, cudaStream_t st) {
   if (per_sm < 1) return cudaErrorInvalidConfiguration;
   long long blocks = (long long)sms * per_sm;
   if (blocks > p.d_out) blocks = p.d_out;
-  kern<<<(unsigned)blocks, nt, smem, st>>>(p);
+  { kern<<<(unsigned)blocks, nt, smem, st>>>(p); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -331,11 +329,6 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
   p.gmagic = ly.g > 1 ? (unsigned)(((1ull << 32) + (unsigned long long)ly.g - 1) / (unsigned long long)ly.g) : 0u;
   const long long d = ly.d_in;
   if (steps_per_col <= 0) return cudaSuccess;   // nothing to do: the counters stay zero, the codes untouched
-  // rows that stream from HBM: two columns in flight per SM
-  if (d > 4096) {
-    const cudaError_t e = launch_cd_pair(p, st);
-    if (e != cudaErrorNotSupported) return e;
-  }
   // short rows (up to 8 KB) are quickest as plain loads into registers; longer ones as bulk copies into
   // shared memory
   if (d > 2048) {
@@ -419,7 +412,7 @@ cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned
   CdParams p{};
   p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
   p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
-  cd_verify_kernel<<<(unsigned)ly.d_out, 128, 0, st>>>(p);
+  { cd_verify_kernel<<<(unsigned)ly.d_out, 128, 0, st>>>(p); count_launch(); }
   return cudaGetLastError();
 }
 

@@ -10,58 +10,26 @@
 // did not: the SM tracks only so many outstanding misses), the sweep starts on the first piece
 // while the others are still landing, and the row no longer occupies 32 registers per thread.
 //
-// Waits on the copy barriers are bounded; when one runs out the kernel records
-// kFlagWaitTimeout in the device status word and carries on (its results are then void).
-#include <cstdlib>
-
+// Waits on the copy barriers are bounded by a cycle count.  A thread whose wait runs out enters the
+// argmin with a key that no real move can have; the whole team sees it after the exchange, starts no
+// further step or column, waits (bounded) for the copies still in flight, records kFlagWaitTimeout
+// in the device status word and returns.
+#include "async_copy.cuh"
 #include "cd_params.cuh"
 #include "cd_sweep.cuh"
 
 namespace cdq {
 namespace {
 
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr long long kWaitCycles = 400ll * 1000 * 1000;   // about 0.2 s
+constexpr unsigned kAbortKey = 0u;    // below the key of every real move (a move's key is at most 0x7FFFFFFF)
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait; false if it ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-// 1-D bulk copy global -> this CTA's shared memory; bytes % 16 == 0, both addresses 16-byte aligned.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
 // NCH chunk slots per thread; the team covers ceil(d_in / 4) <= NT * NCH chunks.
 template <int NCH, int MAXNT, int MINB, int SMODE>
 __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
-  // chunk slots per bulk copy: the 896 x 4 team (rows of up to 57 KB) is quickest with the whole row in one
-  // copy (322 ms against 333 with two and 350 with four on a C3-shaped layer), the 768 x 6 team (74 KB rows,
-  // 24 coordinates per thread) with one copy per slot (616 ms against 640 with twelve, 626 with three, 651 with two and 731 with one);
-  // the 256 x 8 teams of the columns in between, two per SM, again with one copy for the row (d_in = 8192:
-  // 105 ms against 137 with eight copies), and so the 256 x 4 teams of d_in <= 4096
+  // chunk slots per bulk copy: one copy for the whole row, except for the 768 x 6 team of the longest
+  // rows (74 KB), which is quicker with one copy per slot
   constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : ((NCH == 8 && MAXNT == 256) ? 8 : ((NCH == 4 && MAXNT == 256) ? 4 : 1));
   constexpr int NP = NCH / PS;                              // bulk copies per row
   __shared__ __align__(8) unsigned long long s_bar[NP];
@@ -95,7 +63,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   if (tid == 0) {
 #pragma unroll
     for (int k = 0; k < NP; ++k) mbar_init(smem_u32(&s_bar[k]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   // bytes of the row piece behind chunk slot k (0 when the slot lies past the row)
   auto piece_bytes = [&](int k) -> uint32_t {
@@ -103,15 +71,15 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     return hi > lo ? (uint32_t)(hi - lo) * 16u : 0u;
   };
   __syncthreads();
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // zero fill before the first copy lands
+  fence_proxy_async_smem();  // zero fill before the first copy lands
 
   unsigned long long my_committed = 0, my_converged = 0;
   double my_dsum = 0.0;
   uint32_t phase = 0;   // parity of the copy barriers for the next sweep
   int xbuf = 0;
-  bool timed_out = false;
+  bool aborted = false;
 
-  for (;;) {
+  while (!aborted) {
     __syncthreads();  // everyone is done with the previous column
     if (tid == 0) s_col = atomicAdd(&p.ctr->next_col, 1);
     __syncthreads();
@@ -153,7 +121,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     }
 
     // ---- descent ----
-    // The first sweep only scores: it "applies" a step of size zero along row 0.
+    // The first sweep only scores: it "applies" a step of size zero along row 0.  (T >= 1: the launcher
+    // skips the kernel for an empty budget.)
     long long step = 0;
     long long rowoff = 0;
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
@@ -178,6 +147,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       }
       SweepBest sb;
       sb.init();
+      bool timed_out = false;
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         const int cs = tid + NT * k;
@@ -186,7 +156,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         float a, ia;
         chunk_scale(k, a, ia);
         if ((k % PS) == 0 && (exact || NT * k < nchs)) {
-          if (!mbar_wait(smem_u32(&s_bar[k / PS]), phase)) timed_out = true;
+          if (!timed_out && !mbar_wait_cycles(smem_u32(&s_bar[k / PS]), phase, kWaitCycles)) {
+            timed_out = true;
+            atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
+          }
         }
         const float4 rv = row_s[cs];
         double gk[4] = {g[4 * k], g[4 * k + 1], g[4 * k + 2], g[4 * k + 3]};
@@ -194,11 +167,11 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
       }
       phase ^= 1u;
-      if (step >= p.T) break;
 
       // ---- team-wide argmin: (decrease, lowest coordinate, lowest level) ----
       unsigned key, packed;
       sweep_candidate(sb, tid, key, packed);
+      if (timed_out) { key = kAbortKey; packed = 0u; }
       unsigned m = __reduce_min_sync(0xFFFFFFFFu, key);
       unsigned w = __reduce_min_sync(0xFFFFFFFFu, key == m ? packed : kNoMove);
       if (nwarps > 1) {
@@ -210,6 +183,16 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         xbuf ^= 1;
       } else {
         __syncwarp();
+      }
+      if (m == kAbortKey) {   // a copy never landed: wait (bounded) for the pieces of this row, then give up
+        if (tid == 0) {
+#pragma unroll
+          for (int k = 0; k < NP; ++k)
+            if (piece_bytes(k)) mbar_wait_cycles(smem_u32(&s_bar[k]), phase ^ 1u, kWaitCycles);
+          atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
+        }
+        aborted = true;
+        break;
       }
       if (m == kNoMove) { done = true; break; }  // no move lowers the loss
       const int kstar = (int)(w >> 21), tstar = (int)((w >> 11) & 1023u), vstar = (int)((w >> 9) & 3u);
@@ -230,8 +213,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       c2 = 2.0 * ((double)astar * (double)dri);
       rowoff = (long long)istar * p.d_in;
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
-      ++step;
+      // budget used up: the gradient after the last move is never read, so no sweep follows it
+      if (++step >= p.T) break;
     }
+    if (aborted) break;
     if (tid == 0) {
       if (done) ++my_converged;
       my_committed += (unsigned long long)step;
@@ -249,7 +234,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     }
   }
 
-  if (timed_out) atomicExch(p.status, (int)kFlagWaitTimeout);
   if (tid == 0) {
     if (my_dsum != 0.0) atomicAdd(&p.ctr->delta_sum, my_dsum);
     if (my_committed) atomicAdd(&p.ctr->committed, my_committed);
@@ -280,7 +264,7 @@ cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
   if (per_sm < 1) return cudaErrorInvalidConfiguration;
   long long blocks = (long long)sms * per_sm;
   if (blocks > p.d_out) blocks = p.d_out;
-  kern<<<(unsigned)blocks, nt, smem, st>>>(p);
+  { kern<<<(unsigned)blocks, nt, smem, st>>>(p); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -303,13 +287,8 @@ cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st) {
   if (ch <= 128) return launch_mode<2, 64, 8>(p, team(ch, 2), st);
   if (ch <= 1024) return launch_mode<4, 256, 3>(p, team(ch, 4), st);
   if (ch <= 2048) return launch_mode<8, 256, 2>(p, team(ch, 8), st);
-  static const int wide = [] { const char* e = getenv("CDQ_CD_WIDE"); return e ? atoi(e) : 1; }();
-  if (wide) {
-    if (ch <= 3584) return launch_mode<4, 896, 1>(p, team(ch, 4), st);
-    if (ch <= 4608) return launch_mode<6, 768, 1>(p, team(ch, 6), st);
-  }
-  if (ch <= 3584) return launch_mode<8, 448, 1>(p, team(ch, 8), st);
-  if (ch <= 4608) return launch_mode<8, 576, 1>(p, team(ch, 8), st);
+  if (ch <= 3584) return launch_mode<4, 896, 1>(p, team(ch, 4), st);
+  if (ch <= 4608) return launch_mode<6, 768, 1>(p, team(ch, 6), st);
   return cudaErrorNotSupported;
 }
 

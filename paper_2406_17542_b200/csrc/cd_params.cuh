@@ -49,8 +49,4 @@ inline int cd_scale_mode(const CdParams& p, int nt) {
 // plain kernel).
 cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st);
 
-// cd_kernel_pair.cu: rows streamed from HBM with two columns in flight per SM (d_in > 4096).
-// Returns cudaErrorNotSupported when the shape has no such configuration.
-cudaError_t launch_cd_pair(const CdParams& p, cudaStream_t st);
-
 }  // namespace cdq

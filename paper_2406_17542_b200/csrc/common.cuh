@@ -21,6 +21,11 @@ int* device_status_word();  // device address of the status word (per process)
 // Text returned by cdq_last_error_detail().
 void set_error_detail(const char* text);
 
+// Every kernel launch of the library goes through this count (cdq_kernel_launches()).
+void count_launch();
+// H is read with 16-byte vector loads and bulk copies by every consumer after cdq_hessian.
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 // Resolved problem description shared by the launchers.
 struct Layer {
   const float* H;
@@ -102,7 +107,6 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
 // gemm_i8.cu); the losses of the OWC search (round-to-nearest residuals) need ~1e-7 relative.
 constexpr int kTcGradNH = 6, kTcGradNE = 5, kTcGradSmax = 9;
 constexpr int kTcLossNH = 4, kTcLossNE = 4, kTcLossSmax = 6;
-bool gemm_tc_enabled();   // false when CDQ_GEMM=simt is set in the environment
 
 // cd_kernel.cu
 struct CdCounters {            // lives in the workspace, zeroed by the launcher

@@ -148,9 +148,9 @@ __global__ void partials_reduce_kernel(const double* __restrict__ part, long lon
 cudaError_t launch_gemm_he(const float* H, long long d_in, long long d_out, const double* E, double* G,
                            long long ldg, double* col_loss, double* part, cudaStream_t st) {
   dim3 grid((unsigned)((d_out + GN - 1) / GN), (unsigned)((d_in + GM - 1) / GM));
-  gemm_he_kernel<<<grid, 256, 0, st>>>(H, d_in, d_out, E, G, ldg, col_loss ? part : nullptr);
+  { gemm_he_kernel<<<grid, 256, 0, st>>>(H, d_in, d_out, E, G, ldg, col_loss ? part : nullptr); count_launch(); }
   if (col_loss)
-    partials_reduce_kernel<<<(unsigned)((d_out + 127) / 128), 128, 0, st>>>(part, (d_in + GM - 1) / GM, d_out, col_loss);
+    { partials_reduce_kernel<<<(unsigned)((d_out + 127) / 128), 128, 0, st>>>(part, (d_in + GM - 1) / GM, d_out, col_loss); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -182,8 +182,8 @@ __global__ void verify_epilogue_kernel(const double* __restrict__ C, const doubl
 cudaError_t launch_gemm_he_verify(const float* H, long long d_in, long long d_out, const double* E, double* C,
                                   double* G, long long ldg, double* col_loss, cudaStream_t st) {
   dim3 grid((unsigned)((d_out + 127) / 128), (unsigned)d_in);
-  gemm_he_verify_kernel<<<grid, 128, 0, st>>>(H, d_in, d_out, E, C);
-  verify_epilogue_kernel<<<(unsigned)((d_out + 127) / 128), 128, 0, st>>>(C, E, d_in, d_out, G, ldg, col_loss);
+  { gemm_he_verify_kernel<<<grid, 128, 0, st>>>(H, d_in, d_out, E, C); count_launch(); }
+  { verify_epilogue_kernel<<<(unsigned)((d_out + 127) / 128), 128, 0, st>>>(C, E, d_in, d_out, G, ldg, col_loss); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -196,7 +196,7 @@ __global__ void sum_f64_kernel(const double* __restrict__ v, long long n, double
 }
 
 cudaError_t launch_sum_f64(const double* v, long long n, double* out, cudaStream_t st) {
-  sum_f64_kernel<<<1, 32, 0, st>>>(v, n, out);
+  { sum_f64_kernel<<<1, 32, 0, st>>>(v, n, out); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(1024) sum_f64_tree_kernel(const double* __rest
 }
 
 cudaError_t launch_sum_f64_tree(const double* v, long long n, double* out, cudaStream_t st) {
-  sum_f64_tree_kernel<<<1, 1024, 0, st>>>(v, n, out);
+  { sum_f64_tree_kernel<<<1, 1024, 0, st>>>(v, n, out); count_launch(); }
   return cudaGetLastError();
 }
 

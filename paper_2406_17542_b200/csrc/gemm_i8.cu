@@ -455,9 +455,9 @@ cudaError_t gemm_tc_prepare_h(const float* H, long long d_in, int nh, void* hbuf
   const long long kp = tc_kpad(d_in);
   signed char* slices = (signed char*)hbuf;
   int* hexp = (int*)((char*)hbuf + align_up((size_t)nh * d_in * kp));
-  i8::row_exp_f32_kernel<<<(unsigned)d_in, 256, 0, st>>>(H, d_in, d_in, hexp);
+  { i8::row_exp_f32_kernel<<<(unsigned)d_in, 256, 0, st>>>(H, d_in, d_in, hexp); count_launch(); }
   dim3 grid((unsigned)((kp + 255) / 256), (unsigned)d_in);
-  i8::slice_h_kernel<<<grid, 256, 0, st>>>(H, d_in, kp, hexp, nh, slices);
+  { i8::slice_h_kernel<<<grid, 256, 0, st>>>(H, d_in, kp, hexp, nh, slices); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -503,10 +503,10 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
   if (e != cudaSuccess) return e;
   {
     dim3 grid((unsigned)((d_out + 255) / 256), (unsigned)((d_in + 255) / 256));
-    col_max_f64_kernel<<<grid, 256, 0, st>>>(E, d_in, d_out, colmax);
-    col_exp_kernel<<<(unsigned)((d_out + 255) / 256), 256, 0, st>>>(colmax, d_out, eexp);
+    { col_max_f64_kernel<<<grid, 256, 0, st>>>(E, d_in, d_out, colmax); count_launch(); }
+    { col_exp_kernel<<<(unsigned)((d_out + 255) / 256), 256, 0, st>>>(colmax, d_out, eexp); count_launch(); }
     dim3 g2((unsigned)((kp + 31) / 32), (unsigned)((d_out + 31) / 32)), b2(32, 8);
-    slice_et_kernel<<<g2, b2, 0, st>>>(E, d_in, d_out, kp, eexp, ne, esl);
+    { slice_et_kernel<<<g2, b2, 0, st>>>(E, d_in, d_out, kp, eexp, ne, esl); count_launch(); }
   }
   Params p{};
   p.M = (int)d_out; p.N = (int)d_in; p.kblocks = (int)(kp / BKB);
@@ -543,11 +543,11 @@ cudaError_t gemm_tc_run(const void* hbuf, int nh, const double* E, long long d_i
   e = cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int ntiles = p.tiles_m * p.tiles_n;
-  gemm_i8_kernel<<<ntiles < sms ? ntiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(map_e, map_h, p);
+  { gemm_i8_kernel<<<ntiles < sms ? ntiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(map_e, map_h, p); count_launch(); }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (col_loss) {
-    dot_reduce_kernel<<<(unsigned)((d_out + 255) / 256), 256, 0, st>>>(dot_part, 2 * p.tiles_n, d_out, 1.0 / scale, col_loss);
+    { dot_reduce_kernel<<<(unsigned)((d_out + 255) / 256), 256, 0, st>>>(dot_part, 2 * p.tiles_n, d_out, 1.0 / scale, col_loss); count_launch(); }
     e = cudaGetLastError();
   }
   return e;

@@ -46,12 +46,12 @@ cudaError_t launch_hessian_verify(const void* X, cdq_dtype xt, long long n, long
                                   double lambda_rel, float* H, double* H64, cudaStream_t st) {
   dim3 block(128), grid((unsigned)((d_in + 127) / 128), (unsigned)d_in);
   if (xt == CDQ_BF16)
-    hessian_verify_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)X, n, d_in, ldx, H64);
+    { hessian_verify_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)X, n, d_in, ldx, H64); count_launch(); }
   else
-    hessian_verify_kernel<float><<<grid, block, 0, st>>>((const float*)X, n, d_in, ldx, H64);
-  if (lambda_rel > 0.0) lambda_verify_kernel<<<1, 32, 0, st>>>(H64, d_in, lambda_rel);
+    { hessian_verify_kernel<float><<<grid, block, 0, st>>>((const float*)X, n, d_in, ldx, H64); count_launch(); }
+  if (lambda_rel > 0.0) { lambda_verify_kernel<<<1, 32, 0, st>>>(H64, d_in, lambda_rel); count_launch(); }
   const long long count = d_in * d_in;
-  round_to_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(H64, H, count);
+  { round_to_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(H64, H, count); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -124,9 +124,9 @@ cudaError_t launch_hessian_simt(const void* X, cdq_dtype xt, long long n, long l
   const unsigned t = (unsigned)((d_in + HT - 1) / HT);
   dim3 grid(t, t), block(256);
   if (xt == CDQ_BF16)
-    hessian_simt_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)X, n, d_in, ldx, accumulate, H);
+    { hessian_simt_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)X, n, d_in, ldx, accumulate, H); count_launch(); }
   else
-    hessian_simt_kernel<float><<<grid, block, 0, st>>>((const float*)X, n, d_in, ldx, accumulate, H);
+    { hessian_simt_kernel<float><<<grid, block, 0, st>>>((const float*)X, n, d_in, ldx, accumulate, H); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -146,7 +146,7 @@ __global__ void lambda_kernel(float* H, long long d_in, double lambda_rel) {
 }
 
 cudaError_t launch_hessian_lambda(float* H, long long d_in, double lambda_rel, double*, cudaStream_t st) {
-  lambda_kernel<<<1, 256, 0, st>>>(H, d_in, lambda_rel);
+  { lambda_kernel<<<1, 256, 0, st>>>(H, d_in, lambda_rel); count_launch(); }
   return cudaGetLastError();
 }
 

@@ -366,7 +366,7 @@ cudaError_t launch_hessian_tc(const void* X, long long n, long long d_in, long l
   p.partials = (float*)ws;
   int2* tiles = (int2*)((char*)ws + align_up((size_t)pl.splits * pl.ntiles * TILE_ELEMS * sizeof(float)));
   p.tiles = tiles;
-  hessian_tile_order_kernel<<<1, 32, 0, st>>>(pl.tiles_m, tiles);
+  { hessian_tile_order_kernel<<<1, 32, 0, st>>>(pl.tiles_m, tiles); count_launch(); }
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
   int dev = 0, sms = 0;
@@ -376,10 +376,10 @@ cudaError_t launch_hessian_tc(const void* X, long long n, long long d_in, long l
   if (e != cudaSuccess) return e;
   const int units = pl.ntiles * pl.splits;
   const int grid = units < sms ? units : sms;
-  hessian_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmap, p);
+  { hessian_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmap, p); count_launch(); }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  hessian_reduce_kernel<<<pl.ntiles, 256, 0, st>>>(p, accumulate, H);
+  { hessian_reduce_kernel<<<pl.ntiles, 256, 0, st>>>(p, accumulate, H); count_launch(); }
   return cudaGetLastError();
 }
 

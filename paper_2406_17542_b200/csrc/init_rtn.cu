@@ -111,7 +111,7 @@ __global__ void residual_kernel(ResidualSrc s, long long d_in, double* __restric
 
 cudaError_t launch_residual_f64(const ResidualSrc& src, long long d_in, double* E, cudaStream_t st) {
   dim3 block(128), grid((unsigned)((src.d_out + 127) / 128), (unsigned)d_in);
-  residual_kernel<<<grid, block, 0, st>>>(src, d_in, E);
+  { residual_kernel<<<grid, block, 0, st>>>(src, d_in, E); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -140,9 +140,9 @@ __global__ void fill_gamma_kernel(float* gamma_out, long long d_out) {
 cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* mn, float* mx, cudaStream_t st) {
   const long long cpg = (ly.g + kChunkRows - 1) / kChunkRows;
   const unsigned bx = (unsigned)((ly.d_out + 127) / 128);
-  minmax_partial_kernel<<<dim3(bx, (unsigned)(ly.ng * cpg)), 128, 0, st>>>(ly.W, ly.wt, ly.d_in, ly.d_out, ly.ldw, ly.g,
-                                                                            cpg, pmn, pmx);
-  minmax_final_kernel<<<dim3(bx, (unsigned)ly.ng), 128, 0, st>>>(pmn, pmx, ly.ng, ly.d_out, cpg, mn, mx);
+  { minmax_partial_kernel<<<dim3(bx, (unsigned)(ly.ng * cpg)), 128, 0, st>>>(ly.W, ly.wt, ly.d_in, ly.d_out, ly.ldw, ly.g,
+                                                                            cpg, pmn, pmx); count_launch(); }
+  { minmax_final_kernel<<<dim3(bx, (unsigned)ly.ng), 128, 0, st>>>(pmn, pmx, ly.ng, ly.d_out, cpg, mn, mx); count_launch(); }
   return cudaGetLastError();
 }
 
@@ -171,7 +171,7 @@ static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n
     w.table = take(sizeof(double) * n_clip * d_out);
     w.E = take(sizeof(double) * d_in * d_out);
     w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
-    w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+    w.tc = mode == CDQ_MODE_FAST && gemm_tc_supported(d_in, d_out);
     w.ldc = (d_in + 3) / 4 * 4;
     if (w.tc) {
       w.C = take(sizeof(double) * d_out * w.ldc);
@@ -200,9 +200,9 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
   float* mx = (float*)(base + L.mx);
   const unsigned bx = (unsigned)((d_out + 127) / 128);
 
-  minmax_partial_kernel<<<dim3(bx, (unsigned)(ng * cpg)), 128, 0, st>>>(ly.W, ly.wt, d_in, d_out, ly.ldw, g, cpg,
-                                                                         pmn, pmx);
-  minmax_final_kernel<<<dim3(bx, (unsigned)ng), 128, 0, st>>>(pmn, pmx, ng, d_out, cpg, mn, mx);
+  { minmax_partial_kernel<<<dim3(bx, (unsigned)(ng * cpg)), 128, 0, st>>>(ly.W, ly.wt, d_in, d_out, ly.ldw, g, cpg,
+                                                                         pmn, pmx); count_launch(); }
+  { minmax_final_kernel<<<dim3(bx, (unsigned)ng), 128, 0, st>>>(pmn, pmx, ng, d_out, cpg, mn, mx); count_launch(); }
 
   const double* gam_col = nullptr;
   if (n_clip > 1) {
@@ -237,13 +237,13 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
         e = launch_gemm_he_verify(ly.H, d_in, d_out, E, part, nullptr, 0, table + (long long)k * d_out, st);
       if (e != cudaSuccess) return e;
     }
-    owc_argmin_kernel<<<bx, 128, 0, st>>>(table, n_clip, d_out, gammas, gcol, gamma_out);
+    { owc_argmin_kernel<<<bx, 128, 0, st>>>(table, n_clip, d_out, gammas, gcol, gamma_out); count_launch(); }
     gam_col = gcol;
   } else if (gamma_out) {
-    fill_gamma_kernel<<<bx, 128, 0, st>>>(gamma_out, d_out);
+    { fill_gamma_kernel<<<bx, 128, 0, st>>>(gamma_out, d_out); count_launch(); }
   }
-  scale_zero_kernel<<<dim3(bx, (unsigned)ng), 128, 0, st>>>(mn, mx, ng, d_out, ly.L, gam_col, scale, zero);
-  rtn_codes_kernel<<<dim3(bx, (unsigned)d_in), 128, 0, st>>>(ly.W, ly.wt, d_in, d_out, ly.ldw, g, ly.L, scale, zero, Q);
+  { scale_zero_kernel<<<dim3(bx, (unsigned)ng), 128, 0, st>>>(mn, mx, ng, d_out, ly.L, gam_col, scale, zero); count_launch(); }
+  { rtn_codes_kernel<<<dim3(bx, (unsigned)d_in), 128, 0, st>>>(ly.W, ly.wt, d_in, d_out, ly.ldw, g, ly.L, scale, zero, Q); count_launch(); }
   return cudaGetLastError();
 }
 

@@ -46,6 +46,7 @@ extern "C" cdq_status cdq_layer_loss_static(const float* H, const void* W, cdq_d
                                             const float* scale, const float* zero, const unsigned char* Q,
                                             double* loss, double* per_col, void* stream) {
   if (!H || !W || !scale || !zero || !Q || !grid || (wt != CDQ_F32 && wt != CDQ_BF16)) return CDQ_ERR_INVALID_ARG;
+  if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
   if (grid->bits < 1 || grid->bits > 8 || grid->group_size < 0) return CDQ_ERR_INVALID_ARG;
   if (d_in < 1 || d_out < 1 || ldw < d_out) return CDQ_ERR_SHAPE;
   if (grid->group_size > 0 && d_in % grid->group_size) return CDQ_ERR_SHAPE;

@@ -388,7 +388,7 @@ static OwcWs owc_ws_layout(long long d_in, long long d_out, long long g, int nk,
   w.col_after = take(sizeof(double) * d_out);
   w.sums = take(sizeof(double) * 2);
   w.ctr = take(sizeof(owc::Counters));
-  w.tc = mode == CDQ_MODE_FAST && gemm_tc_enabled() && gemm_tc_supported(d_in, d_out);
+  w.tc = mode == CDQ_MODE_FAST && gemm_tc_supported(d_in, d_out);
   w.ldg = (d_in + 3) / 4 * 4;
   if (w.tc) {
     w.E = take(sizeof(double) * d_in * d_out);
@@ -452,13 +452,13 @@ cudaError_t launch_owc_cd(const Layer& ly, const cdq_grid_desc& grid, long long 
   const size_t smem = 2 * sizeof(double) * (size_t)ng * nk;
   if (mode == CDQ_MODE_FP64_VERIFY || smem > 160 * 1024) {
     p.Gext = nullptr;
-    owc::owc_cd_kernel<true><<<ctas, owc::NT, 0, st>>>(p);
+    { owc::owc_cd_kernel<true><<<ctas, owc::NT, 0, st>>>(p); count_launch(); }
   } else {
     if (smem > 40 * 1024) {
       e = cudaFuncSetAttribute(owc::owc_cd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
-    owc::owc_cd_kernel<false><<<ctas, owc::NT, smem, st>>>(p);
+    { owc::owc_cd_kernel<false><<<ctas, owc::NT, smem, st>>>(p); count_launch(); }
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

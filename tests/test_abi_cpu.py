@@ -103,6 +103,31 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert lib.cdq_hessian_add_lambda(dummy, 8, -1.0, null) == 1
 
 
+def test_misaligned_hessian_is_rejected_before_any_launch(lib):
+    """H is read with 16-byte vector loads and bulk copies: a pointer 4 bytes off (a view into a larger
+    tensor, say) must be refused by every entry point that takes H, not faulted on."""
+    gd = B.Grid(bits=3).c()
+    owc = B.Grid(bits=3, n_clip=4, clip_lo=0.5, clip_hi=1.0).c()
+    dummy, off4, null = ctypes.c_void_p(256), ctypes.c_void_p(260), None
+    big = 1 << 30
+    assert lib.cdq_hessian(dummy, 0, 16, 8, 8, 0.0, 0, off4, 0, dummy, big, null) == 1
+    assert lib.cdq_init_rtn(dummy, 0, 8, 8, 8, off4, ctypes.byref(owc), dummy, dummy, dummy, null, 0, dummy, big, null) == 1
+    assert lib.cdq_init_owc_cd(dummy, 0, 8, 8, 8, off4, ctypes.byref(owc), 0, dummy, dummy, dummy, null, None, 0,
+                               dummy, big, null) == 1
+    assert lib.cdq_cd_solve(off4, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, 1, 0, None, dummy, big, null) == 1
+    assert lib.cdq_cd_solve_steps(off4, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, 4, 0, None, dummy, big,
+                                  null) == 1
+    assert lib.cdq_bcd_solve(off4, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, 2, 4, 0, 0, None, dummy, big,
+                             null) == 1
+    assert lib.cdq_layer_loss(off4, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, None, null, 0, dummy, big,
+                              null) == 1
+    assert lib.cdq_layer_loss_static(off4, dummy, 0, 8, 8, 8, ctypes.byref(gd), dummy, dummy, dummy, None, null, null) == 1
+    # the diagnostics entry points check their ranges before touching the device
+    assert lib.cdq_debug_expire_wait(0, null) == 1
+    assert lib.cdq_debug_set_device_status(7) == 1
+    assert lib.cdq_kernel_launches() == 0   # nothing above reached a launch
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))

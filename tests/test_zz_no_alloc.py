@@ -3,12 +3,14 @@
 that stops at the first failure has already been through every other test.
 
 Checks, through the C ABI: two calls in a row (the shared scratch keeps the first call's
-contents) give the same result as cdq_layer_loss with a caller workspace, and a layer that
-does not fit in the fixed array is refused with a message."""
+contents) give the same result as cdq_layer_loss with a caller workspace and as the CPU oracle's
+loss from the definition (Eq. 1 with H = X^T X), and a layer that does not fit in the fixed array is
+refused with a message."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2406_17542_b200 import binding as B
 from paper_2406_17542_b200 import inputs
 
@@ -49,6 +51,11 @@ def test_static_scratch_matches_workspace_version_twice():
         results.append((got, want))
         assert abs(got - want) <= RTOL * abs(want)
         np.testing.assert_allclose(cols.cpu().numpy(), want_cols.cpu().numpy(), rtol=RTOL)
+        # the expected value itself: the oracle's loss on the same H, W, grid and codes
+        ref, ref_cols = oracle.layer_loss(H.cpu().numpy(), W.cpu(), scale.cpu().numpy(), zero.cpu().numpy(),
+                                          Q.cpu().numpy(), cfg.group_size)
+        assert abs(got - ref) <= RTOL * abs(ref)
+        np.testing.assert_allclose(cols.cpu().numpy(), ref_cols, rtol=RTOL)
         # and once more on the same layer, without per-column output
         again = B.cdq_layer_loss_static(H, W, grid, scale, zero, Q)
         assert abs(again - want) <= RTOL * abs(want)
