@@ -33,6 +33,12 @@ constexpr int A_BYTES = BM * BK * 2;               // 2 boxes
 constexpr int B_BYTES = BN * BK * 2;               // 4 boxes
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 49152
 constexpr int TILE_ELEMS = BM * BN;
+// K blocks (of BK rows) that one TMEM accumulator takes before the epilogue drains it.  The tensor core's
+// fp32 accumulation truncates, so the error of an entry grows with the number of accumulation steps behind
+// it: with all 131072 rows of a layer in one accumulator the entries came out up to 7e-4 (of sqrt(H_ii H_jj))
+// low, with 262144 rows past the 1e-3 the Hessian is allowed.  256 blocks = 16384 rows per accumulator bound
+// that near 6e-5; the chunks of a tile are added up by the epilogue with round-to-nearest fp32 adds.
+constexpr int KCHUNK = 256;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t SPIN_LIMIT = 1u << 22;
@@ -222,27 +228,31 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, Params p) {
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         const int s = u / p.ntiles;
         const int kb0 = (int)((long long)s * p.kblocks / p.splits), kb1 = (int)((long long)(s + 1) * p.kblocks / p.splits);
-        if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t tmem_d = tmem_base + (uint32_t)buf * BN;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+        // one accumulator takes at most KCHUNK K blocks (see KCHUNK); the epilogue adds the chunks up
+        for (int kc0 = kb0; kc0 < kb1 && ok; kc0 += KCHUNK) {
+          const int kc1 = min(kb1, kc0 + KCHUNK);
+          if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_src = tiles + (uint32_t)stage * STAGE_BYTES;
-          const uint32_t b_src = a_src + A_BYTES;
+          const uint32_t tmem_d = tmem_base + (uint32_t)buf * BN;
+          for (int kb = kc0; kb < kc1; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_src = tiles + (uint32_t)stage * STAGE_BYTES;
+            const uint32_t b_src = a_src + A_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            // 16 rows of X = two 8-row swizzle groups = 2 KB further into every 64-column block
-            const uint64_t adesc = make_desc(a_src + kk * 2048);
-            const uint64_t bdesc = make_desc(b_src + kk * 2048);
-            mma_f16(tmem_d, adesc, bdesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              // 16 rows of X = two 8-row swizzle groups = 2 KB further into every 64-column block
+              const uint64_t adesc = make_desc(a_src + kk * 2048);
+              const uint64_t bdesc = make_desc(b_src + kk * 2048);
+              mma_f16(tmem_d, adesc, bdesc, (kb > kc0 || kk > 0) ? 1u : 0u);
+            }
+            mma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
-          mma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (!ok) break;
+          mma_commit(tfull_bar(buf));       // accumulator complete
+          if (++buf == 2) { buf = 0; tphase ^= 1u; }
         }
-        if (!ok) break;
-        mma_commit(tfull_bar(buf));       // accumulator complete
-        if (++buf == 2) { buf = 0; tphase ^= 1u; }
       }
     }
   } else {
@@ -253,24 +263,35 @@ hessian_tc_kernel(const __grid_constant__ CUtensorMap tmap, Params p) {
     uint32_t tphase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-      if (!mbar_wait(tfull_bar(buf), tphase, abort_flag)) { ok = false; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int s = u / p.ntiles;
+      const int kb0 = (int)((long long)s * p.kblocks / p.splits), kb1 = (int)((long long)(s + 1) * p.kblocks / p.splits);
       float* out = p.partials + (size_t)u * TILE_ELEMS + (size_t)row * BN;
+      for (int kc0 = kb0; kc0 < kb1 && ok; kc0 += KCHUNK) {
+        if (!mbar_wait(tfull_bar(buf), tphase, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const bool first = kc0 == kb0;   // later chunks add to what this thread stored before (round-to-nearest adds)
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), r);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int v = 0; v < 8; ++v)
-          *reinterpret_cast<float4*>(out + c * 32 + v * 4) =
-              make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                          __uint_as_float(r[4 * v + 3]));
+          for (int v = 0; v < 8; ++v) {
+            float4 x = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                   __uint_as_float(r[4 * v + 3]));
+            float4* dst = reinterpret_cast<float4*>(out + c * 32 + v * 4);
+            if (!first) {
+              const float4 y = *dst;
+              x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+            }
+            *dst = x;
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(buf));
+        if (++buf == 2) { buf = 0; tphase ^= 1u; }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
-      if (++buf == 2) { buf = 0; tphase ^= 1u; }
     }
   }
 
