@@ -43,6 +43,15 @@ __device__ __forceinline__ bool mbar_wait_cycles(uint32_t bar, uint32_t parity, 
   } while (clock64() - t0 < cycles);
   return false;
 }
+// The same with the 32-bit clock (fewer registers in a hot loop); cycles < 2^31.
+__device__ __forceinline__ bool mbar_wait_clock32(uint32_t bar, uint32_t parity, unsigned cycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned t0 = (unsigned)clock();
+  do {
+    if (mbar_try_wait(bar, parity)) return true;
+  } while ((unsigned)clock() - t0 < cycles);
+  return false;
+}
 // Generic-proxy writes to shared memory (a zero fill, say) before the copy engine touches it.
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

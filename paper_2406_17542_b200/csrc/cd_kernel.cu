@@ -161,8 +161,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
     }
 
     // ---- descent ----
-    // The first sweep only scores: it "applies" a step of size zero along row 0.  (T >= 1: the launcher
-    // skips the kernel for an empty budget.)
+    // The first sweep only scores: it "applies" a step of size zero along row 0.
     long long step = 0;
     const float* rp = p.H;
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
@@ -202,6 +201,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
         g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
       }
 
+      if (step >= p.T) break;
+
       // ---- team-wide argmin: (decrease, lowest coordinate, lowest level) ----
       unsigned key, packed;
       sweep_candidate(sb, tid, key, packed);
@@ -236,8 +237,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
       c2 = 2.0 * ((double)astar * (double)dri);
       rp = p.H + (long long)istar * d_in;
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
-      // budget used up: the gradient after the last move is never read, so no sweep follows it
-      if (++step >= p.T) break;
+      ++step;
     }
     if (tid == 0) {
       if (done) ++my_converged;

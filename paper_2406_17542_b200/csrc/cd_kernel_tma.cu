@@ -21,7 +21,7 @@
 namespace cdq {
 namespace {
 
-constexpr long long kWaitCycles = 400ll * 1000 * 1000;   // about 0.2 s
+constexpr unsigned kWaitCycles = 400u * 1000u * 1000u;   // about 0.2 s
 constexpr unsigned kAbortKey = 0u;    // below the key of every real move (a move's key is at most 0x7FFFFFFF)
 
 // NCH chunk slots per thread; the team covers ceil(d_in / 4) <= NT * NCH chunks.
@@ -121,8 +121,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     }
 
     // ---- descent ----
-    // The first sweep only scores: it "applies" a step of size zero along row 0.  (T >= 1: the launcher
-    // skips the kernel for an empty budget.)
+    // The first sweep only scores: it "applies" a step of size zero along row 0.
     long long step = 0;
     long long rowoff = 0;
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
@@ -156,10 +155,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         float a, ia;
         chunk_scale(k, a, ia);
         if ((k % PS) == 0 && (exact || NT * k < nchs)) {
-          if (!timed_out && !mbar_wait_cycles(smem_u32(&s_bar[k / PS]), phase, kWaitCycles)) {
-            timed_out = true;
-            atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
-          }
+          if (!mbar_wait_clock32(smem_u32(&s_bar[k / PS]), phase, kWaitCycles)) timed_out = true;
         }
         const float4 rv = row_s[cs];
         double gk[4] = {g[4 * k], g[4 * k + 1], g[4 * k + 2], g[4 * k + 3]};
@@ -167,6 +163,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
       }
       phase ^= 1u;
+      if (step >= p.T) {   // budget used up (this sweep only brought the gradient up to date)
+        if (timed_out) atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
+        break;
+      }
 
       // ---- team-wide argmin: (decrease, lowest coordinate, lowest level) ----
       unsigned key, packed;
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         if (tid == 0) {
 #pragma unroll
           for (int k = 0; k < NP; ++k)
-            if (piece_bytes(k)) mbar_wait_cycles(smem_u32(&s_bar[k]), phase ^ 1u, kWaitCycles);
+            if (piece_bytes(k)) mbar_wait_clock32(smem_u32(&s_bar[k]), phase ^ 1u, kWaitCycles);
           atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
         }
         aborted = true;
@@ -213,8 +213,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       c2 = 2.0 * ((double)astar * (double)dri);
       rowoff = (long long)istar * p.d_in;
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
-      // budget used up: the gradient after the last move is never read, so no sweep follows it
-      if (++step >= p.T) break;
+      ++step;
     }
     if (aborted) break;
     if (tid == 0) {
