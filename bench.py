@@ -114,12 +114,12 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def algorithmic_bytes_cd(cfg, committed: int) -> float:
-    """Descent kernel: one fp32 row of H per committed move, plus per-column state in and out
-    (fp64 gradient in, codes in and out, scales)."""
+def algorithmic_bytes_cd(cfg, committed: int, row_bytes: float = 4.0) -> float:
+    """Descent kernel: one row of H per committed move (fp32, or bf16 with --rows16), plus per-column state in
+    and out (fp64 gradient in, codes in and out, scales)."""
     ng = cfg.d_in // cfg.group_size if cfg.group_size else 1
     per_col = 8 * cfg.d_in + 2 * cfg.d_in + 4 * ng
-    return committed * 4.0 * cfg.d_in + cfg.d_out * float(per_col)
+    return committed * row_bytes * cfg.d_in + cfg.d_out * float(per_col)
 
 
 def run_oracle_sample(cfg, X, W, n_rows: int, n_cols: int) -> dict:
@@ -260,7 +260,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         Q0 = Q.clone() if (times is not None and parity_cols > 0 and not host) else None   # (a copy, not a kernel of the library)
         budget = cfg.d_in // args.budget_div if args.budget_div > 0 else None
         stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
-                               steps_per_col=budget if args.block == 1 else None)
+                               steps_per_col=budget if args.block == 1 else None, rows16=args.rows16)
         if args.block == 2:  # the paper starts BCD from the greedy solution
             cd_stats = stats
             stats = B.cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, budget or cfg.d_in, seed=cfg.seed, ws=ws)
@@ -327,13 +327,13 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
     acc = cfg.scaled(d_out=W.shape[1], n=X.shape[0])   # what this rank worked on (the whole layer unless --shard)
     mean = lambda v: sum(v) / len(v)
     cd_ms = mean(times["cd_kernel"])
-    alg_bytes = algorithmic_bytes_cd(acc, committed)
+    alg_bytes = algorithmic_bytes_cd(acc, committed, 2.0 if args.rows16 else 4.0)
     if args.block == 2:  # two rows per move at most, and one H_im per pair and step
         alg_bytes += committed * 4.0 * cfg.d_in + stats["steps"] * 2.0 * cfg.d_in
     achieved = alg_bytes / (cd_ms * 1e-3) / 1e9
     h_bytes = 4.0 * cfg.d_in * cfg.d_in
     hbm_served = h_bytes > L2_BYTES
-    kernel = descent_kernel_name(cfg, args.block)
+    kernel = descent_kernel_name(cfg, args.block) + ("<bf16 rows>" if args.rows16 else "")
     per_move = NCU_TRAFFIC_PER_MOVE.get((kernel, cfg.d_in))
     if hbm_served:
         roofline = {"kernel": kernel, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -383,7 +383,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
         rec["e2e"] = {"value": committed_all / (total_ms_e2e / steps * 1e-3), "unit": UNIT,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": total_ms_e2e / steps}
-    if parity_cols > 0 and keep and args.block == 1 and args.init == "rtn" and args.budget_div == 0:
+    if parity_cols > 0 and keep and args.block == 1 and args.init == "rtn" and args.budget_div == 0 and not args.rows16:
         rec["parity"] = parity_in_run(B, cfg, grid, keep["H"], keep["W"], keep["scale"], keep["zero"], keep["Q0"],
                                       keep["Q"], keep["gamma"], keep["per"], parity_cols)
     rec["_inputs"] = (X, W)
@@ -395,7 +395,8 @@ def workload_name(cfg, args) -> str:
             f"bits={cfg.bits} group={cfg.group_size or 'per-channel'} n_clip={cfg.n_clip} passes={cfg.passes}"
             + (" init=OWC-CD" if args.init == "owc_cd" else "")
             + (f" budget=d_in/{args.budget_div}" if args.budget_div > 0 else "")
-            + (" descent=CD then BCD(k=2)" if args.block == 2 else ""))
+            + (" descent=CD then BCD(k=2)" if args.block == 2 else "")
+            + (" rows=bf16" if args.rows16 else ""))
 
 
 def main():
@@ -422,6 +423,9 @@ def main():
     ap.add_argument("--init", default="rtn", choices=["rtn", "owc_cd"],
                     help="grid stage: cdq_init_rtn (MinMax / OWC as the config says) or cdq_init_owc_cd (Algorithm 3; "
                          "configs with a clipping grid)")
+    ap.add_argument("--rows16", action="store_true",
+                    help="the descent reads its rows from a bf16 copy of H (cdq_cd_solve_rows16): 2 d_in bytes per move; the "
+                         "reported loss is on the true H; no in-run parity (tests/test_rows16_gpu.py holds it)")
     ap.add_argument("--shard", action="store_true",
                     help="share ONE layer out over the ranks (strong scaling): rows of X per rank for the Hessian with one "
                          "all-reduce, columns of W per rank after it; the default gives every rank its own layer (weak)")
@@ -484,7 +488,7 @@ def main():
     gc.collect()
     torch.cuda.empty_cache()
     if world == 1 and not args.no_other_configs and not profiling_case and args.block == 1 and args.init == "rtn" \
-            and args.budget_div == 0 and not args.shard:
+            and args.budget_div == 0 and not args.shard and not args.rows16:
         others = {}
         for name in ("C1", "C2", "C4"):
             if name == cfg.name:

@@ -74,7 +74,8 @@ typedef enum {
   CDQ_CALL_CD_SOLVE = 2,
   CDQ_CALL_LAYER_LOSS = 3,
   CDQ_CALL_INIT_OWC_CD = 4,
-  CDQ_CALL_BCD_SOLVE = 5   /* n: steps per column */
+  CDQ_CALL_BCD_SOLVE = 5,  /* n: steps per column */
+  CDQ_CALL_CD_SOLVE_ROWS16 = 6
 } cdq_call;
 
 /* Quantization grid (paper: c in "Notation"; group size g in the sub-channel
@@ -238,6 +239,25 @@ cdq_status cdq_bcd_solve(const float* H, const void* W, cdq_dtype wt, long long 
                          const float* zero, unsigned char* Q, int block, long long steps_per_col,
                          unsigned long long seed, cdq_mode mode, cdq_cd_stats* stats, void* ws,
                          size_t ws_bytes, void* stream);
+
+/*
+ * The greedy descent with 2-byte rows (paper: the appendix on run time puts the cost of a step in the
+ * gather of the Hessian row and its scatter into the gradient, and speeds the method up by taking fewer
+ * steps; this variant halves the bytes of each step instead, at a stated cost in the loss).
+ * The update g += 2 d H[i*, :] reads row i* from a bf16 copy of H that the call builds in its workspace
+ * (round to nearest even); H_ii stays fp32 everywhere (the scores, and the moved coordinate's own entry of
+ * the row).  The call is therefore exactly cdq_cd_solve_steps on the matrix H' with H'_ij = bf16(H_ij) for
+ * i != j and H'_ii = H_ii: the starting gradient, the tracked loss in `stats` and the picks all refer to
+ * H'.  What that costs on the true objective is for the caller to measure with cdq_layer_loss on H.
+ *   Arguments as for cdq_cd_solve_steps; production arithmetic only.
+ *   Workspace: cdq_workspace_bytes(CDQ_CALL_CD_SOLVE_ROWS16, ...) = that of cdq_cd_solve plus 6 d_in^2 bytes.
+ *   CDQ_ERR_UNSUPPORTED unless d_in > 2048, d_in % 8 == 0 and the group size is a multiple of 4 (shorter rows
+ *   are served from L2 and gain nothing from fewer bytes).
+ */
+cdq_status cdq_cd_solve_rows16(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                               long long ldw, const cdq_grid_desc* grid, const float* scale, const float* zero,
+                               unsigned char* Q, long long steps_per_col, cdq_cd_stats* stats, void* ws,
+                               size_t ws_bytes, void* stream);
 
 /*
  * Layer loss sum_j e_j^T H e_j with e = W_hat - W (paper: Eq. 1 written with

@@ -22,9 +22,10 @@ STATUS_NAMES = {0: "CDQ_OK", 1: "CDQ_ERR_INVALID_ARG", 2: "CDQ_ERR_SHAPE", 3: "C
 CDQ_F32, CDQ_BF16 = 0, 1
 MODE_FAST, MODE_FP64_VERIFY = 0, 1
 CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD, CALL_BCD_SOLVE = 0, 1, 2, 3, 4, 5
+CALL_CD_SOLVE_ROWS16 = 6
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
+EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_cd_solve_rows16", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version",
            "cdq_kernel_launches", "cdq_debug_expire_wait", "cdq_debug_set_device_status"]
@@ -102,6 +103,8 @@ def load():
                                   ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_cd_solve_steps.restype = ci
     lib.cdq_cd_solve_steps.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
+    lib.cdq_cd_solve_rows16.restype = ci
+    lib.cdq_cd_solve_rows16.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_layer_loss.restype = ci
     lib.cdq_layer_loss.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ctypes.POINTER(ctypes.c_double), vp, ci, vp, sz, vp]
     lib.cdq_layer_loss_static.restype = ci
@@ -237,9 +240,10 @@ def cdq_init_owc_cd(W: torch.Tensor, grid: Grid, H: torch.Tensor, steps: int = 0
 
 def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,
                  Q: torch.Tensor, passes: int, mode="fast", want_stats: bool = True, ws: Workspace | None = None,
-                 steps_per_col: int | None = None):
+                 steps_per_col: int | None = None, rows16: bool = False):
     """Greedy coordinate descent on every column; Q is updated in place.  Returns the stats dict (or None).
-    With steps_per_col the budget is that many steps per column (cdq_cd_solve_steps) instead of passes * d_in."""
+    With steps_per_col the budget is that many steps per column (cdq_cd_solve_steps) instead of passes * d_in.
+    rows16: the update reads its rows from a bf16 copy of H (cdq_cd_solve_rows16)."""
     _need_cuda(H, W, scale, zero, Q)
     d_in, d_out = W.shape
     assert H.shape == (d_in, d_in) and H.is_contiguous() and H.dtype == torch.float32
@@ -248,6 +252,17 @@ def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tens
     gd = grid.c()
     stats = cdq_cd_stats()
     ws = ws or _default_ws
+    if rows16:
+        wptr, wbytes = ws.get(workspace_bytes(CALL_CD_SOLVE_ROWS16, 0, d_in, d_out, grid, mode), W.device)
+        st = load().cdq_cd_solve_rows16(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), ctypes.byref(gd),
+                                        scale.data_ptr(), zero.data_ptr(), Q.data_ptr(),
+                                        int(passes * d_in if steps_per_col is None else steps_per_col),
+                                        ctypes.byref(stats) if want_stats else None, wptr, wbytes, _stream())
+        _check(st, "cdq_cd_solve_rows16")
+        if not want_stats:
+            return None
+        return {"steps": stats.steps, "committed": stats.committed, "columns_converged": stats.columns_converged,
+                "loss_before": stats.loss_before, "loss_after": stats.loss_after, "kernel_ms": stats.kernel_ms}
     wptr, wbytes = ws.get(workspace_bytes(CALL_CD_SOLVE, 0, d_in, d_out, grid, mode), W.device)
     fn = load().cdq_cd_solve if steps_per_col is None else load().cdq_cd_solve_steps
     st = fn(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), ctypes.byref(gd),

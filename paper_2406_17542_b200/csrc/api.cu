@@ -80,12 +80,13 @@ Layer make_layer(const float* H, const void* W, cdq_dtype wt, long long d_in, lo
 
 // Workspace of cdq_cd_solve / cdq_layer_loss.
 struct SolveWs {
-  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, hbuf, ebuf, bcd_tab, total;
+  size_t E, G, Qt, hdiag, half_inv, part, col_loss, scalars, hbuf, ebuf, bcd_tab, h16, hr, total;
   long long ldg, d_pad;
   bool tc;        // H E on the int8 tensor cores
   int nh, ne, smax;
 };
-SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd, long long bcd_steps = 0) {
+SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool with_cd, long long bcd_steps = 0,
+                        bool rows16 = false) {
   SolveWs w{};
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
@@ -111,6 +112,10 @@ SolveWs solve_ws_layout(long long d_in, long long d_out, cdq_mode mode, bool wit
   w.col_loss = take(sizeof(double) * d_out);
   w.scalars = take(256);  // [0]: loss sum; [64..): CdCounters
   if (bcd_steps > 0 && mode == CDQ_MODE_FAST) w.bcd_tab = take(bcd_table_bytes(d_in, bcd_steps));
+  if (rows16) {
+    w.h16 = take(sizeof(__nv_bfloat16) * (size_t)d_in * d_in);
+    w.hr = take(sizeof(float) * (size_t)d_in * d_in);
+  }
   w.total = off;
   return w;
 }
@@ -256,6 +261,9 @@ size_t cdq_workspace_bytes(cdq_call which, long long n, long long d_in, long lon
     case CDQ_CALL_LAYER_LOSS:
       if (d_out < 1) return 0;
       return solve_ws_layout(d_in, d_out, mode, false).total;
+    case CDQ_CALL_CD_SOLVE_ROWS16:
+      if (d_out < 1) return 0;
+      return solve_ws_layout(d_in, d_out, mode, true, 0, true).total;
   }
   return 0;
 }
@@ -337,7 +345,7 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
 static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
                                 const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
                                 long long steps_per_col, int block, unsigned long long seed, cdq_mode mode,
-                                cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream) {
+                                cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream, bool rows16 = false) {
   if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || steps_per_col < 0)
     return CDQ_ERR_INVALID_ARG;
   if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
@@ -349,12 +357,22 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   s = check_grid(grid, d_in);
   if (s != CDQ_OK) return s;
   if (block > 1 && steps_per_col > 65535) return CDQ_ERR_UNSUPPORTED;
-  const SolveWs L = solve_ws_layout(d_in, d_out, mode, true, block > 1 ? steps_per_col : 0);
+  if (rows16) {
+    const long long g = grid->group_size > 0 ? grid->group_size : d_in;
+    if (mode != CDQ_MODE_FAST || block != 1 || !cd_rows16_supported(d_in, g)) return CDQ_ERR_UNSUPPORTED;
+  }
+  const SolveWs L = solve_ws_layout(d_in, d_out, mode, true, block > 1 ? steps_per_col : 0, rows16);
   s = check_ws(ws, ws_bytes, L.total);
   if (s != CDQ_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
-  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, scale, zero);
   char* base = (char*)ws;
+  const __nv_bfloat16* H16 = nullptr;
+  if (rows16) {   // everything below works on H with its off-diagonal entries rounded to bf16
+    CDQ_CUDA(launch_round_rows_bf16(H, d_in, (__nv_bfloat16*)(base + L.h16), (float*)(base + L.hr), st));
+    H16 = (const __nv_bfloat16*)(base + L.h16);
+    H = (const float*)(base + L.hr);
+  }
+  Layer ly = make_layer(H, W, wt, d_in, d_out, ldw, grid, scale, zero);
   double* E = (double*)(base + L.E);
   double* G = (double*)(base + L.G);
   unsigned char* Qt = (unsigned char*)(base + L.Qt);
@@ -393,7 +411,7 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   } else if (fast_cd) {
     CDQ_CUDA(launch_diag(H, d_in, L.d_pad, hdiag, half_inv, st));
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
-    CDQ_CUDA(launch_cd_fast(ly, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, ctr, st));
+    CDQ_CUDA(launch_cd_fast(ly, H16, G, L.ldg, Qt, L.ldg, hdiag, half_inv, steps_per_col, ctr, st));
   } else {
     if (stats) CDQ_CUDA(cudaEventRecord(ev0, st));
     CDQ_CUDA(launch_cd_verify(ly, G, L.ldg, Qt, L.ldg, steps_per_col, ctr, st));
@@ -433,6 +451,14 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
                               size_t ws_bytes, void* stream) {
   return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, 1, 0ull, mode, stats, ws,
                        ws_bytes, stream);
+}
+
+cdq_status cdq_cd_solve_rows16(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                               long long ldw, const cdq_grid_desc* grid, const float* scale, const float* zero,
+                               unsigned char* Q, long long steps_per_col, cdq_cd_stats* stats, void* ws,
+                               size_t ws_bytes, void* stream) {
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, 1, 0ull, CDQ_MODE_FAST, stats, ws,
+                       ws_bytes, stream, true);
 }
 
 cdq_status cdq_bcd_solve(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,

@@ -318,11 +318,33 @@ bool cd_fast_supported(long long d_in, long long g) {
   return d_in >= 1 && d_in <= 18432 && (g == d_in || (g & 3) == 0);
 }
 
-cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
-                           const float* hdiag, const float* hs, long long steps_per_col,
+// The bf16-row descent runs in the kernel that stages its rows through shared memory: d_in > 2048 (shorter rows
+// are L2-served and gain nothing), rows 16-byte aligned as bf16.
+bool cd_rows16_supported(long long d_in, long long g) {
+  return cd_fast_supported(d_in, g) && d_in > 2048 && (d_in & 7) == 0;
+}
+
+__global__ void round_rows_bf16_kernel(const float* __restrict__ H, long long d_in, __nv_bfloat16* __restrict__ H16,
+                                       float* __restrict__ Hr) {
+  const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (idx >= d_in * d_in) return;
+  const float h = H[idx];
+  const __nv_bfloat16 b = __float2bfloat16_rn(h);
+  H16[idx] = b;
+  Hr[idx] = (idx / d_in == idx % d_in) ? h : __bfloat162float(b);
+}
+
+cudaError_t launch_round_rows_bf16(const float* H, long long d_in, __nv_bfloat16* H16, float* Hr, cudaStream_t st) {
+  const long long total = d_in * d_in;
+  { round_rows_bf16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(H, d_in, H16, Hr); count_launch(); }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cd_fast(const Layer& ly, const __nv_bfloat16* H16, double* G, long long ldg, unsigned char* Qt,
+                           long long ldq, const float* hdiag, const float* hs, long long steps_per_col,
                            CdCounters* ctr, cudaStream_t st) {
   CdParams p{};
-  p.H = ly.H; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
+  p.H = ly.H; p.H16 = H16; p.d_in = ly.d_in; p.d_out = ly.d_out; p.G = G; p.ldg = ldg; p.Qt = Qt; p.ldq = ldq; p.scale = ly.scale;
   p.hdiag = hdiag; p.hs = hs; p.g = ly.g; p.ng = ly.ng; p.L = ly.L; p.T = steps_per_col; p.ctr = ctr;
   p.status = device_status_word();
   if (!p.status) return cudaErrorInvalidSymbol;
@@ -335,6 +357,7 @@ cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned c
     const cudaError_t e = launch_cd_tma(p, st);
     if (e != cudaErrorNotSupported) return e;
   }
+  if (H16) return cudaErrorNotSupported;
   auto team = [&](int ept) { return (int)(((d + ept - 1) / ept + 31) / 32 * 32); };
   if (d <= 512) return launch_cd_shape<2, 64, 8>(p, team(8), st);
   if (d <= 4096) return launch_cd_shape<4, 256, 3>(p, team(16), st);

@@ -25,7 +25,9 @@ constexpr unsigned kWaitCycles = 400u * 1000u * 1000u;   // about 0.2 s
 constexpr unsigned kAbortKey = 0u;    // below the key of every real move (a move's key is at most 0x7FFFFFFF)
 
 // NCH chunk slots per thread; the team covers ceil(d_in / 4) <= NT * NCH chunks.
-template <int NCH, int MAXNT, int MINB, int SMODE>
+// ROW16: the rows come from a bf16 copy of H (half the bytes per move); the row's own diagonal element is
+// replaced by the exact H_ii, so the iteration is the descent on H with its off-diagonal entries rounded to bf16.
+template <int NCH, int MAXNT, int MINB, int SMODE, bool ROW16>
 __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
   // chunk slots per bulk copy: one copy for the whole row, except for the 768 x 6 team of the longest
@@ -42,8 +44,9 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   const bool exact = nchs == NT * NCH;
   const float top = kMagic + (float)p.L;
 
-  float4* row_s = reinterpret_cast<float4*>(dyn_smem);                  // [NCH * NT]
-  float2* ag_s = reinterpret_cast<float2*>(row_s + (size_t)NCH * NT);  // [ag_count] (a, 1/a), grouped modes
+  constexpr int CHB = ROW16 ? 8 : 16;                                   // bytes of a chunk of 4 row entries
+  unsigned char* row_s = dyn_smem;                                      // [NCH * NT] chunks
+  float2* ag_s = reinterpret_cast<float2*>(row_s + (size_t)NCH * NT * CHB);  // [ag_count] (a, 1/a), grouped modes
   auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
   const int g4 = SMODE == kGroupFast ? (int)(p.g >> 2) : 1;
   const float2* ag_mine = ag_s + (SMODE == kGroupFast ? tid / g4 : 0);
@@ -59,7 +62,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   };
 
   // slots past the end of the row stay zero: no copy ever writes there
-  for (int t = tid; t < NCH * NT; t += NT) row_s[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int t = tid; t < NCH * NT * CHB / 8; t += NT) reinterpret_cast<uint2*>(row_s)[t] = make_uint2(0u, 0u);
   if (tid == 0) {
 #pragma unroll
     for (int k = 0; k < NP; ++k) mbar_init(smem_u32(&s_bar[k]), 1);
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   // bytes of the row piece behind chunk slot k (0 when the slot lies past the row)
   auto piece_bytes = [&](int k) -> uint32_t {
     const int lo = NT * PS * k, hi = min(NT * PS * (k + 1), nchs);
-    return hi > lo ? (uint32_t)(hi - lo) * 16u : 0u;
+    return hi > lo ? (uint32_t)(hi - lo) * (uint32_t)CHB : 0u;
   };
   __syncthreads();
   fence_proxy_async_smem();  // zero fill before the first copy lands
@@ -124,6 +127,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     // The first sweep only scores: it "applies" a step of size zero along row 0.
     long long step = 0;
     long long rowoff = 0;
+    [[maybe_unused]] bool fix_diag = false;   // ROW16: this thread owns the coordinate of the move being applied ...
+    [[maybe_unused]] int kprev = 0, vprev = 0;   // ... in chunk slot kprev, position vprev
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
     double col_dsum = 0.0;
     bool done = frozen;
@@ -132,7 +137,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       // column prologue): the copies may overwrite it
       // piece k is requested by the first lane of warp k (by thread 0 when the team has fewer warps)
       {
-        const float* src = p.H + rowoff;
+        const unsigned char* src = ROW16 ? reinterpret_cast<const unsigned char*>(p.H16 + rowoff)
+                                         : reinterpret_cast<const unsigned char*>(p.H + rowoff);
 #pragma unroll
         for (int k = 0; k < NP; ++k) {
           const bool issuer = nwarps >= NP ? (warp == k && lane == 0) : tid == 0;
@@ -140,7 +146,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
           if (issuer && bytes) {
             const uint32_t bar = smem_u32(&s_bar[k]);
             mbar_expect_tx(bar, bytes);
-            bulk_load(smem_u32(row_s + (size_t)NT * PS * k), src + (size_t)NT * PS * k * 4, bytes, bar);
+            bulk_load(smem_u32(row_s + (size_t)NT * PS * k * CHB), src + (size_t)NT * PS * k * CHB, bytes, bar);
           }
         }
       }
@@ -157,7 +163,18 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         if ((k % PS) == 0 && (exact || NT * k < nchs)) {
           if (!mbar_wait_clock32(smem_u32(&s_bar[k / PS]), phase, kWaitCycles)) timed_out = true;
         }
-        const float4 rv = row_s[cs];
+        float4 rv;
+        if constexpr (ROW16) {
+          const uint2 rr = reinterpret_cast<const uint2*>(row_s)[cs];
+          rv = make_float4(__uint_as_float(rr.x << 16), __uint_as_float(rr.x & 0xFFFF0000u),
+                           __uint_as_float(rr.y << 16), __uint_as_float(rr.y & 0xFFFF0000u));
+          if (fix_diag && k == kprev) {   // this thread holds the coordinate that moved: its own entry of the row is H_ii
+            rv.x = vprev == 0 ? hd.x : rv.x; rv.y = vprev == 1 ? hd.y : rv.y;
+            rv.z = vprev == 2 ? hd.z : rv.z; rv.w = vprev == 3 ? hd.w : rv.w;
+          }
+        } else {
+          rv = reinterpret_cast<const float4*>(row_s)[cs];
+        }
         double gk[4] = {g[4 * k], g[4 * k + 1], g[4 * k + 2], g[4 * k + 3]};
         sweep_chunk<SMODE>(gk, rv, hd, hs, qp[k], c2, a, ia, top, k, sb);
         g[4 * k] = gk[0]; g[4 * k + 1] = gk[1]; g[4 * k + 2] = gk[2]; g[4 * k + 3] = gk[3];
@@ -202,6 +219,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         if (tid == 0) atomicExch(p.status, (int)kFlagBadIndex);
         istar = 0;
       }
+      if constexpr (ROW16) { fix_diag = tid == tstar; kprev = kstar; vprev = vstar; }
       if (tid == tstar) {
         const unsigned dq = (unsigned)dri << (8 * vstar);
 #pragma unroll
@@ -240,18 +258,18 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   }
 }
 
-template <int NCH, int MAXNT, int MINB, int SMODE>
+template <int NCH, int MAXNT, int MINB, int SMODE, bool ROW16>
 cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
   p.ag_count = (int)p.ng;
   if (SMODE == kGroupFast) {
     const int g4 = (int)(p.g >> 2), slots = (nt * NCH + g4 - 1) / g4;
     if (slots > p.ag_count) p.ag_count = slots;
   }
-  auto kern = cd_tma_kernel<NCH, MAXNT, MINB, SMODE>;
+  auto kern = cd_tma_kernel<NCH, MAXNT, MINB, SMODE, ROW16>;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const size_t smem = (size_t)NCH * nt * sizeof(float4) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
+  const size_t smem = (size_t)NCH * nt * (ROW16 ? 8 : 16) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
   cudaError_t e;
   if (smem > 48 * 1024) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -270,9 +288,15 @@ cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
 template <int NCH, int MAXNT, int MINB>
 cudaError_t launch_mode(const CdParams& p, int nt, cudaStream_t st) {
   const int smode = cd_scale_mode(p, nt);
-  if (smode == kPerChannel) return launch_cfg<NCH, MAXNT, MINB, kPerChannel>(p, nt, st);
-  if (smode == kGroupFast) return launch_cfg<NCH, MAXNT, MINB, kGroupFast>(p, nt, st);
-  if (smode == kGroupAny) return launch_cfg<NCH, MAXNT, MINB, kGroupAny>(p, nt, st);
+  if (p.H16) {
+    if (smode == kPerChannel) return launch_cfg<NCH, MAXNT, MINB, kPerChannel, true>(p, nt, st);
+    if (smode == kGroupFast) return launch_cfg<NCH, MAXNT, MINB, kGroupFast, true>(p, nt, st);
+    if (smode == kGroupAny) return launch_cfg<NCH, MAXNT, MINB, kGroupAny, true>(p, nt, st);
+    return cudaErrorNotSupported;
+  }
+  if (smode == kPerChannel) return launch_cfg<NCH, MAXNT, MINB, kPerChannel, false>(p, nt, st);
+  if (smode == kGroupFast) return launch_cfg<NCH, MAXNT, MINB, kGroupFast, false>(p, nt, st);
+  if (smode == kGroupAny) return launch_cfg<NCH, MAXNT, MINB, kGroupAny, false>(p, nt, st);
   return cudaErrorNotSupported;
 }
 
@@ -281,6 +305,7 @@ cudaError_t launch_mode(const CdParams& p, int nt, cudaStream_t st) {
 cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st) {
   if (p.d_in & 3) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(p.H) & 15) != 0) return cudaErrorNotSupported;
+  if (p.H16 && ((p.d_in & 7) != 0 || (reinterpret_cast<uintptr_t>(p.H16) & 15) != 0)) return cudaErrorNotSupported;
   const long long ch = p.d_in >> 2;
   auto team = [&](long long chunks, int nch) { return (int)((chunks + nch - 1) / nch + 31) / 32 * 32; };
   if (ch <= 128) return launch_mode<2, 64, 8>(p, team(ch, 2), st);

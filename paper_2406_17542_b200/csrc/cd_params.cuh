@@ -7,6 +7,7 @@ namespace cdq {
 
 struct CdParams {
   const float* H;
+  const __nv_bfloat16* H16;   // bf16 copy of H for the rows of the update (NULL: fp32 rows)
   long long d_in, d_out;
   double* G;            // [d_out, ldg]
   long long ldg;

@@ -122,9 +122,14 @@ long long cd_fast_pad(long long d_in);      // padded length of hdiag / hs
 bool cd_fast_supported(long long d_in, long long g);
 // hdiag = H_ii, hs = 0.5 / H_ii
 cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* hs, cudaStream_t st);
-cudaError_t launch_cd_fast(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
-                           const float* hdiag, const float* hs, long long steps_per_col,
+// H16 (may be NULL): bf16 copy of H for the rows of the update; cudaErrorNotSupported if the shape has no such kernel
+cudaError_t launch_cd_fast(const Layer& ly, const __nv_bfloat16* H16, double* G, long long ldg, unsigned char* Qt,
+                           long long ldq, const float* hdiag, const float* hs, long long steps_per_col,
                            CdCounters* ctr, cudaStream_t st);
+bool cd_rows16_supported(long long d_in, long long g);   // shapes whose descent can read bf16 rows
+// H16 = bf16(H) and Hr = the fp32 matrix the bf16-row descent works on: off-diagonal entries rounded to bf16
+// (round to nearest even), diagonal exact
+cudaError_t launch_round_rows_bf16(const float* H, long long d_in, __nv_bfloat16* H16, float* Hr, cudaStream_t st);
 cudaError_t launch_cd_verify(const Layer& ly, double* G, long long ldg, unsigned char* Qt, long long ldq,
                              long long steps_per_col, CdCounters* ctr, cudaStream_t st);
 // bcd_kernel.cu: random blocks of two coordinates (Algorithm 2 / 5)

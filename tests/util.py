@@ -103,7 +103,7 @@ OWC_TIE = 1e-7   # relative gap of two clipping strengths' column losses below w
 
 
 def compare_with_oracle(cfg, H32, Hd, Wd, cols, g, scale_d, zero_d, Q0_d, Q_d, gamma_d, per_d, budget, label="",
-                        code_agree=0.999, loss_rtol=1e-4):
+                        code_agree=0.999, loss_rtol=1e-4, rows16=False):
     """Production-mode result of the library on columns `cols` of a layer against the oracle on the same columns
     with the same fp32 H: grid and starting codes bit for bit, final codes up to audited fp32 near-tie forks, the
     summed column losses within loss_rtol.  With a clipping search, a column whose clipping strength differs is
@@ -132,8 +132,11 @@ def compare_with_oracle(cfg, H32, Hd, Wd, cols, g, scale_d, zero_d, Q0_d, Q_d, g
     ref = oracle.cd_solve(H32, Wc, cfg.bits, init["scale"], init["zero"], init["Q"], budget, cfg.group_size)
     _, per_ref = oracle.layer_loss(H32, Wc, init["scale"], init["zero"], ref["Q"], cfg.group_size)
     kt = ct[torch.from_numpy(keep).to(dev)]
-    replay = lib_replay(Hd, Wd[:, kt].contiguous(), g, scale_d[:, kt].contiguous(), zero_d[:, kt].contiguous(),
-                        Q0_d[:, kt].contiguous())
+    Wk_d, sk_d, zk_d = Wd[:, kt].contiguous(), scale_d[:, kt].contiguous(), zero_d[:, kt].contiguous()
+    solve = None
+    if rows16:   # the replays must be the same kind of run (Hd is then the matrix the caller handed to the library)
+        solve = lambda Q, t: B.cdq_cd_solve(Hd, Wk_d, g, sk_d, zk_d, Q, 0, steps_per_col=t, rows16=True)
+    replay = lib_replay(Hd, Wk_d, g, sk_d, zk_d, Q0_d[:, kt].contiguous(), solve=solve)
     Wk = Wc[:, torch.from_numpy(keep)]
     out = check_codes_with_fork_audit(H32, Wk, cfg, init["scale"][:, keep], init["zero"][:, keep], init["Q"][:, keep],
                                       ref["Q"][:, keep], Q_d[:, kt].cpu().numpy(), budget, replay, code_agree, label)
