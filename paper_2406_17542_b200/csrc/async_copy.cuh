@@ -52,6 +52,21 @@ __device__ __forceinline__ bool mbar_wait_clock32(uint32_t bar, uint32_t parity,
   } while ((unsigned)clock() - t0 < cycles);
   return false;
 }
+// Bounded wait for the pipelines whose roles (producer, MMA issuer, epilogue) give up together: false if the
+// wait ran out (the flag is then set) or another role has already given up.
+__device__ __forceinline__ bool mbar_wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   uint32_t spin_limit) {
+  for (uint32_t it = 0; it < spin_limit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+// tcgen05.commit: the mbarrier is arrived on once the MMAs issued so far have completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
 // Generic-proxy writes to shared memory (a zero fill, say) before the copy engine touches it.
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -5,10 +5,6 @@
 // (fp64) and scores the best move of every coordinate (fp32) -- the body of the loop of
 // Algorithm 1 of the paper, with its scan over the levels replaced by the clamped rounding of the parabola's vertex
 //   r = clamp(rint(q - g / (2 a H_ii)), 0, L).
-// (Variants that were measured and dropped: a chunk-level running minimum with the winner
-// worked out afterwards, a packed fp64 min carrying score and identity, and an integer-pipe
-// fp64 -> fp32 truncation, and the packed f32x2 arithmetic of sm_100 for the fp32 part; each made
-// the step slower or no faster on B200.)
 #pragma once
 
 #include "cd_params.cuh"

@@ -21,6 +21,7 @@
 // device status word, lets the other roles drain, frees its TMEM and returns.
 #include <cuda.h>
 
+#include "async_copy.cuh"
 #include "common.cuh"
 
 namespace cdq {
@@ -52,36 +53,9 @@ struct Params {
   int* status;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the wait ran out or another role has already given up.
+// Bounded wait of this pipeline's roles (see async_copy.cuh).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
+  return mbar_wait_or_abort(bar, parity, abort_flag, SPIN_LIMIT);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -110,9 +84,6 @@ __device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t adesc, uint64_
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
       : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -332,11 +303,16 @@ static Plan make_plan(long long n, long long d_in) {
   for (int tm = 0; tm < pl.tiles_m; ++tm) nt += tm / 2 + 1;
   pl.ntiles = nt;
   pl.kblocks = (int)((n + BK - 1) / BK);
-  // aim for about two units per SM so that the epilogue of one overlaps the MMAs of the next
-  int splits = (2 * 148 + nt - 1) / nt;
-  if (splits > 16) splits = 16;
-  if (splits > pl.kblocks) splits = pl.kblocks;
-  if (splits < 1) splits = 1;
+  // K-splits: the units (tile x split) run in waves of one per SM; pick the split count whose waves cost
+  // least -- ceil(units / SMs) waves of kblocks / splits K blocks each, plus a fixed cost per unit
+  // (pipeline fill, the epilogue that nothing overlaps) of about 16 K blocks
+  int splits = 1;
+  long long best = -1;
+  for (int s = 1; s <= 16 && s <= pl.kblocks; ++s) {
+    const long long waves = ((long long)nt * s + 147) / 148;
+    const long long cost = waves * ((pl.kblocks + s - 1) / s + 16);
+    if (best < 0 || cost * 100 < best * 97) { best = cost; splits = s; }   // more partial tiles only for a real gain
+  }
   pl.splits = splits;
   return pl;
 }
