@@ -242,7 +242,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
     pinned_out: list = []
     keep: dict = {}
 
-    def one_step(host: bool, times: dict | None = None):
+    def one_step(host: bool, times: dict | None = None, last: bool = False):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
         ev[0].record()
         Xd = Xh.to(dev, non_blocking=True) if host else X
@@ -257,7 +257,9 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         else:
             scale, zero, Q, gamma = B.cdq_init_rtn(Wd, grid, H=H if cfg.n_clip > 1 else None, ws=ws)
         ev[3].record()
-        Q0 = Q.clone() if (times is not None and parity_cols > 0 and not host) else None   # (a copy, not a kernel of the library)
+        # the last timed step keeps what the in-run parity check needs (earlier steps must not: a held H would make
+        # the next step allocate a fresh one inside the timed region)
+        Q0 = Q.clone() if (last and parity_cols > 0 and not host) else None   # (a copy, not a kernel of the library)
         budget = cfg.d_in // args.budget_div if args.budget_div > 0 else None
         stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
                                steps_per_col=budget if args.block == 1 else None, rows16=args.rows16)
@@ -300,10 +302,10 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         d2h = 0
         multi.barrier(world)
         launches0 = lib.cdq_kernel_launches()
-        for _ in range(steps):
+        for it in range(steps):
             flush.fill_(1)           # evict L2 between timed iterations (not timed)
             torch.cuda.synchronize()
-            stats, loss, d2h = one_step(host, times)
+            stats, loss, d2h = one_step(host, times, last=it == steps - 1)
         launches = lib.cdq_kernel_launches() - launches0
         multi.barrier(world)
         return times, stats, loss, d2h, launches

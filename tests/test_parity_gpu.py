@@ -142,19 +142,21 @@ def test_hessian_tensor_core_path(n, d_in):
     Hc = H.cpu().numpy()
     if d_in <= 1200:
         H64, _ = oracle.hessian(X)
-        assert rel_fro(Hc, H64) <= 1e-5          # bf16 products are exact in fp32; only summation error
+        assert rel_fro(Hc, H64) <= 3e-5          # bf16 products are exact in fp32; only summation error
     rng = np.random.default_rng(n)
     rows = rng.integers(0, d_in, 4096); cols = rng.integers(0, d_in, 4096)
     want = oracle.hessian_entries(X, rows, cols)
     got = Hc[rows, cols].astype(np.float64)
     scale = np.sqrt(oracle.hessian_entries(X, rows, rows) * oracle.hessian_entries(X, cols, cols))
-    assert np.max(np.abs(got - want) / scale) <= 1e-5
+    # the tensor core's fp32 accumulation truncates: the error grows with the rows behind one accumulator
+    # (here up to 4096: ~1.3e-5; the library cuts the chains at 16384 rows, ~7e-5 -- tests/test_hessian_scale_gpu.py)
+    assert np.max(np.abs(got - want) / scale) <= 3e-5
     assert np.array_equal(Hc, Hc.T)
     # accumulate over two row chunks == one call
     half = (n // 2) // 8 * 8
     H2 = B.cdq_hessian(Xd[:half])
     H2 = B.cdq_hessian(Xd[half:], accumulate=True, out=H2)
-    assert rel_fro(H2.cpu().numpy(), Hc) <= 1e-5
+    assert rel_fro(H2.cpu().numpy(), Hc) <= 3e-5
 
 
 @pytest.mark.parametrize("mode", ["verify", "fast"])
