@@ -24,7 +24,10 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Calls only enqueue work, except where a host result is returned
  *     (cdq_cd_solve with stats != NULL, cdq_layer_loss with loss != NULL):
- *     those synchronise `stream` before returning.
+ *     those synchronise `stream` before returning.  cdq_init_rtn with a clipping
+ *     search of four or more strengths in the production mode synchronises `stream`
+ *     once in the middle (it reads back how many columns each strength is still a
+ *     candidate for, see there).
  *   - Errors are returned as status codes; nothing aborts or throws.
  *     Arguments are validated before any launch.  A device-side wait that
  *     exceeds its bound is reported as CDQ_ERR_TIMEOUT by the next call that
@@ -140,6 +143,10 @@ cdq_status cdq_hessian_add_lambda(float* H, long long d_in, float lambda_rel, vo
  *   scale,zero [d_in/g, d_out] fp32 out.
  *   Q          [d_in, d_out] u8 out.
  *   gamma_out  [d_out] fp32 out, chosen clipping strength; may be NULL.
+ * FAST, layers of at least 256 x 128: the column losses are products on the int8 tensor cores.  All
+ * strengths are first screened with six slice-pair products; a strength within 2e-4 of a column's smallest
+ * screened loss stays a candidate and gets the thirteen-pair loss (~1e-8 relative); the argmin is taken over
+ * the candidates.  The candidate counts go through the host: one synchronisation of `stream`.
  * The rounding decision is taken in fp64 in both modes.
  */
 cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,

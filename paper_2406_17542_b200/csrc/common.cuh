@@ -78,7 +78,9 @@ struct ResidualSrc {
   const void* W; cdq_dtype wt; long long ldw;
   const float* scale; const float* zero; const unsigned char* Q;  // codes path
   const float* mn; const float* mx; double gamma; int L; int use_gamma;  // OWC path
-  long long g, d_out;
+  long long g, d_out;      // d_out: columns of the layer (the width of W's companions scale, zero, Q, mn, mx)
+  const int* col_idx;      // NULL: E has a column for every layer column; else E column c is layer column col_idx[c] ...
+  long long n_cols;        // ... and E is [d_in, n_cols]
 };
 cudaError_t launch_residual_f64(const ResidualSrc& src, long long d_in, double* E, cudaStream_t st);
 

@@ -84,9 +84,11 @@ __global__ void rtn_codes_kernel(const void* __restrict__ W, cdq_dtype wt, long 
 // Residual E[i][j] = (a q + b) - w in fp64, either from stored codes or, for the OWC search,
 // from min/max and a clipping strength (codes formed on the fly, never stored).
 __global__ void residual_kernel(ResidualSrc s, long long d_in, double* __restrict__ E) {
-  const long long j = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  const long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // column of E
   const long long i = blockIdx.y;
-  if (j >= s.d_out) return;
+  const long long width = s.col_idx ? s.n_cols : s.d_out;
+  if (c >= width) return;
+  const long long j = s.col_idx ? (long long)s.col_idx[c] : c;            // column of the layer
   const long long t = i / s.g;
   const double w = load_w(s.W, s.wt, i * s.ldw + j);
   double a, b, q;
@@ -106,11 +108,12 @@ __global__ void residual_kernel(ResidualSrc s, long long d_in, double* __restric
     b = (double)s.zero[t * s.d_out + j];
     q = (double)s.Q[i * s.d_out + j];
   }
-  E[i * s.d_out + j] = __dadd_rn(__dadd_rn(__dmul_rn(a, q), b), -w);
+  E[i * width + c] = __dadd_rn(__dadd_rn(__dmul_rn(a, q), b), -w);
 }
 
 cudaError_t launch_residual_f64(const ResidualSrc& src, long long d_in, double* E, cudaStream_t st) {
-  dim3 block(128), grid((unsigned)((src.d_out + 127) / 128), (unsigned)d_in);
+  const long long width = src.col_idx ? src.n_cols : src.d_out;
+  dim3 block(128), grid((unsigned)((width + 127) / 128), (unsigned)d_in);
   { residual_kernel<<<grid, block, 0, st>>>(src, d_in, E); count_launch(); }
   return cudaGetLastError();
 }
@@ -129,6 +132,70 @@ __global__ void owc_argmin_kernel(const double* __restrict__ table, int n_clip, 
   }
   gam_col[j] = gammas[bk];
   if (gamma_out) gamma_out[j] = (float)gammas[bk];
+}
+
+// ---- screening of the clipping search (production mode, tensor-core losses) ----
+// The losses of all clipping strengths are first formed cheaply (six slice-pair products instead of thirteen);
+// a strength stays a candidate of a column if its screened loss is within kScreenBand of the column's smallest.
+// Only candidates get the thirteen-pair loss, and the argmin is taken over those: the same result as the full
+// table as long as the screening error stays inside the band.  The screen keeps three 7-bit slices of the
+// residual: the slicing truncates, and a clipped weight leaves a residual many times the typical one, so with
+// two slices (2^-14 of the column's largest residual) the screened loss was off by up to 6e-4 and picked another
+// strength on a C4-shaped layer; with three slices the error is below ~1e-5 and the band leaves a factor of 20.
+constexpr double kScreenBand = 2e-4;
+constexpr int kScreenNE = 3, kScreenSmax = 4;   // pairs (1,1) (1,2) (2,1) (1,3) (2,2) (3,1)
+
+// mask[k][j] = 1 for candidates; the table starts at +inf everywhere.
+__global__ void owc_candidates_kernel(const double* __restrict__ screen, int n_clip, long long d_out,
+                                      unsigned char* __restrict__ mask, double* __restrict__ table) {
+  const long long j = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (j >= d_out) return;
+  double best = screen[j];
+  for (int k = 1; k < n_clip; ++k) best = fmin(best, screen[(long long)k * d_out + j]);
+  const double lim = best + kScreenBand * fabs(best);
+  for (int k = 0; k < n_clip; ++k) {
+    mask[(long long)k * d_out + j] = screen[(long long)k * d_out + j] <= lim ? 1 : 0;
+    table[(long long)k * d_out + j] = __longlong_as_double(0x7FF0000000000000ll);
+  }
+}
+
+// One CTA per clipping strength: its candidate columns in ascending order, padded by repeating the last one to a
+// multiple of 128 (at least 128: the tensor-core product wants that many columns); cnt[k] = padded count (0: none).
+__global__ void __launch_bounds__(1024) owc_compact_kernel(const unsigned char* __restrict__ mask, long long d_out,
+                                                           int* __restrict__ idx, int* __restrict__ cnt) {
+  __shared__ int s_scan[1024];
+  __shared__ int s_base;
+  const int k = blockIdx.x, tid = threadIdx.x;
+  const unsigned char* m = mask + (long long)k * d_out;
+  int* out = idx + (long long)k * (d_out + 128);
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (long long j0 = 0; j0 < d_out; j0 += 1024) {
+    const long long j = j0 + tid;
+    const int f = (j < d_out && m[j]) ? 1 : 0;
+    s_scan[tid] = f;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {
+      const int v = tid >= o ? s_scan[tid - o] : 0;
+      __syncthreads();
+      s_scan[tid] += v;
+      __syncthreads();
+    }
+    if (f) out[s_base + s_scan[tid] - 1] = (int)j;
+    __syncthreads();
+    if (tid == 0) s_base += s_scan[1023];
+    __syncthreads();
+  }
+  const int n = s_base;
+  const int padded = n == 0 ? 0 : (n + 127) / 128 * 128;
+  for (int t = n + tid; t < padded; t += 1024) out[t] = out[n - 1];
+  if (tid == 0) cnt[k] = padded;
+}
+
+__global__ void owc_scatter_kernel(const double* __restrict__ loss_c, const int* __restrict__ idx, int n,
+                                   double* __restrict__ table_row) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < n) table_row[idx[c]] = loss_c[c];   // padding repeats a column with its own value
 }
 
 __global__ void fill_gamma_kernel(float* gamma_out, long long d_out) {
@@ -151,7 +218,8 @@ cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* 
 //   OWC only : gammas [n_clip] f64, gam_col [d_out] f64, table [n_clip, d_out] f64,
 //              E [d_in, d_out] f64, loss partials (FAST) or the product H E (VERIFY)
 struct InitWs {
-  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, total;
+  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, screen, mask, idx, cnt, loss_c, total;
+  bool screened;    // cheap losses first, exact ones for the near-tied strengths only
   bool tc;          // losses on the int8 tensor cores
   long long ldc;
 };
@@ -169,14 +237,22 @@ static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n
     w.gammas = take(sizeof(double) * n_clip);
     w.gam_col = take(sizeof(double) * d_out);
     w.table = take(sizeof(double) * n_clip * d_out);
-    w.E = take(sizeof(double) * d_in * d_out);
+    w.E = take(sizeof(double) * d_in * (d_out + 128));
     w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
     w.tc = mode == CDQ_MODE_FAST && gemm_tc_supported(d_in, d_out);
     w.ldc = (d_in + 3) / 4 * 4;
     if (w.tc) {
-      w.C = take(sizeof(double) * d_out * w.ldc);
+      w.C = take(sizeof(double) * (d_out + 128) * w.ldc);
       w.hbuf = take(gemm_tc_h_bytes(d_in, kTcLossNH));
-      w.ebuf = take(gemm_tc_e_bytes(d_in, d_out, kTcLossNE));
+      w.ebuf = take(gemm_tc_e_bytes(d_in, d_out + 128, kTcLossNE));
+      w.screened = n_clip >= 4;
+      if (w.screened) {
+        w.screen = take(sizeof(double) * n_clip * d_out);
+        w.mask = take((size_t)n_clip * d_out);
+        w.idx = take(sizeof(int) * (size_t)n_clip * (d_out + 128));
+        w.cnt = take(sizeof(int) * n_clip);
+        w.loss_c = take(sizeof(double) * (d_out + 128));
+      }
     }
   }
   w.total = off;
@@ -221,6 +297,45 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
       e = gemm_tc_prepare_h(ly.H, d_in, kTcLossNH, base + L.hbuf, st);
       if (e != cudaSuccess) return e;
     }
+    if (L.screened) {
+      double* screen = (double*)(base + L.screen);
+      unsigned char* mask = (unsigned char*)(base + L.mask);
+      int* idx = (int*)(base + L.idx);
+      int* cnt = (int*)(base + L.cnt);
+      double* loss_c = (double*)(base + L.loss_c);
+      for (int k = 0; k < n_clip; ++k) {   // screening
+        ResidualSrc src{};
+        src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
+        src.mn = mn; src.mx = mx; src.gamma = hg[k]; src.L = ly.L; src.use_gamma = 1;
+        src.g = g; src.d_out = d_out;
+        e = launch_residual_f64(src, d_in, E, st);
+        if (e != cudaSuccess) return e;
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, d_out, kScreenNE, kScreenSmax, 1.0, (double*)(base + L.C), L.ldc,
+                        screen + (long long)k * d_out, base + L.ebuf, st);
+        if (e != cudaSuccess) return e;
+      }
+      { owc_candidates_kernel<<<bx, 128, 0, st>>>(screen, n_clip, d_out, mask, table); count_launch(); }
+      { owc_compact_kernel<<<(unsigned)n_clip, 1024, 0, st>>>(mask, d_out, idx, cnt); count_launch(); }
+      int hcnt[256];
+      e = cudaMemcpyAsync(hcnt, cnt, sizeof(int) * n_clip, cudaMemcpyDeviceToHost, st);
+      if (e != cudaSuccess) return e;
+      e = cudaStreamSynchronize(st);   // the sizes of the exact products are decided on the host
+      if (e != cudaSuccess) return e;
+      for (int k = 0; k < n_clip; ++k) {
+        if (hcnt[k] <= 0) continue;
+        const int* idx_k = idx + (long long)k * (d_out + 128);
+        ResidualSrc src{};
+        src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
+        src.mn = mn; src.mx = mx; src.gamma = hg[k]; src.L = ly.L; src.use_gamma = 1;
+        src.g = g; src.d_out = d_out; src.col_idx = idx_k; src.n_cols = hcnt[k];
+        e = launch_residual_f64(src, d_in, E, st);
+        if (e != cudaSuccess) return e;
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, hcnt[k], kTcLossNE, kTcLossSmax, 1.0, (double*)(base + L.C), L.ldc,
+                        loss_c, base + L.ebuf, st);
+        if (e != cudaSuccess) return e;
+        { owc_scatter_kernel<<<(unsigned)((hcnt[k] + 255) / 256), 256, 0, st>>>(loss_c, idx_k, hcnt[k], table + (long long)k * d_out); count_launch(); }
+      }
+    } else
     for (int k = 0; k < n_clip; ++k) {
       ResidualSrc src{};
       src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
