@@ -126,30 +126,30 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     // ---- descent ----
     // The first sweep only scores: it "applies" a step of size zero along row 0.
     long long step = 0;
-    long long rowoff = 0;
     [[maybe_unused]] bool fix_diag = false;   // ROW16: this thread owns the coordinate of the move being applied ...
     [[maybe_unused]] int kprev = 0, vprev = 0;   // ... in chunk slot kprev, position vprev
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
     double col_dsum = 0.0;
     bool done = frozen;
-    while (!done) {
-      // every thread is past its reads of the previous row (the barrier of the argmin, or of the
-      // column prologue): the copies may overwrite it
-      // piece k is requested by the first lane of warp k (by thread 0 when the team has fewer warps)
-      {
-        const unsigned char* src = ROW16 ? reinterpret_cast<const unsigned char*>(p.H16 + rowoff)
-                                         : reinterpret_cast<const unsigned char*>(p.H + rowoff);
+    // Requests row `off / d_in` of H: piece k by the first lane of warp k (by thread 0 when the team has fewer warps).
+    // Called when every thread is past its reads of the previous row (behind the barrier of the argmin, or of the
+    // column prologue), and as early as the row is known: what follows the argmin overlaps with the copy.
+    auto request_row = [&](long long off) {
+      const unsigned char* src = ROW16 ? reinterpret_cast<const unsigned char*>(p.H16 + off)
+                                       : reinterpret_cast<const unsigned char*>(p.H + off);
 #pragma unroll
-        for (int k = 0; k < NP; ++k) {
-          const bool issuer = nwarps >= NP ? (warp == k && lane == 0) : tid == 0;
-          const uint32_t bytes = piece_bytes(k);
-          if (issuer && bytes) {
-            const uint32_t bar = smem_u32(&s_bar[k]);
-            mbar_expect_tx(bar, bytes);
-            bulk_load(smem_u32(row_s + (size_t)NT * PS * k * CHB), src + (size_t)NT * PS * k * CHB, bytes, bar);
-          }
+      for (int k = 0; k < NP; ++k) {
+        const bool issuer = nwarps >= NP ? (warp == k && lane == 0) : tid == 0;
+        const uint32_t bytes = piece_bytes(k);
+        if (issuer && bytes) {
+          const uint32_t bar = smem_u32(&s_bar[k]);
+          mbar_expect_tx(bar, bytes);
+          bulk_load(smem_u32(row_s + (size_t)NT * PS * k * CHB), src + (size_t)NT * PS * k * CHB, bytes, bar);
         }
       }
+    };
+    if (!done) request_row(0);
+    while (!done) {
       SweepBest sb;
       sb.init();
       bool timed_out = false;
@@ -219,6 +219,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         if (tid == 0) atomicExch(p.status, (int)kFlagBadIndex);
         istar = 0;
       }
+      request_row((long long)istar * p.d_in);
       if constexpr (ROW16) { fix_diag = tid == tstar; kprev = kstar; vprev = vstar; }
       if (tid == tstar) {
         const unsigned dq = (unsigned)dri << (8 * vstar);
@@ -229,7 +230,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       float astar = 1.f;
       if (SMODE != kPerChannel) astar = ag_s[group_of((unsigned)istar)].x;
       c2 = 2.0 * ((double)astar * (double)dri);
-      rowoff = (long long)istar * p.d_in;
       if (tid == 0) col_dsum += (double)__uint_as_float(~m);
       ++step;
     }
