@@ -262,19 +262,27 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         # the next step allocate a fresh one inside the timed region)
         Q0 = Q.clone() if (last and parity_cols > 0 and not host) else None   # (a copy, not a kernel of the library)
         budget = cfg.d_in // args.budget_div if args.budget_div > 0 else None
-        stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
-                               steps_per_col=budget if args.block == 1 else None, rows16=args.rows16)
-        if args.block == 2:  # the paper starts BCD from the greedy solution
-            cd_stats = stats
-            stats = B.cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, budget or cfg.d_in, seed=cfg.seed, ws=ws)
-            stats["cd_kernel_ms_before_bcd"] = cd_stats["kernel_ms"]
-            stats["loss_after_cd"] = cd_stats["loss_after"]
-        ev[4].record()
         want_cols = Q0 is not None
-        loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws, per_col=want_cols)
         per = None
-        if want_cols:
-            loss, per = loss
+        if args.block == 1 and not args.rows16:
+            # the descent returns the loss of its result (half the dot product of residual and final gradient)
+            res = B.cdq_cd_solve_with_loss(H, Wd, grid, scale, zero, Q, budget or cfg.passes * cfg.d_in, ws=ws,
+                                           per_col=want_cols)
+            stats, loss = res[0], res[1]
+            per = res[2] if want_cols else None
+            ev[4].record()
+        else:
+            stats = B.cdq_cd_solve(H, Wd, grid, scale, zero, Q, cfg.passes, ws=ws,
+                                   steps_per_col=budget if args.block == 1 else None, rows16=args.rows16)
+            if args.block == 2:  # the paper starts BCD from the greedy solution
+                cd_stats = stats
+                stats = B.cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, budget or cfg.d_in, seed=cfg.seed, ws=ws)
+                stats["cd_kernel_ms_before_bcd"] = cd_stats["kernel_ms"]
+                stats["loss_after_cd"] = cd_stats["loss_after"]
+            ev[4].record()
+            loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws, per_col=want_cols)
+            if want_cols:
+                loss, per = loss
         if host:   # results back into pinned host buffers (allocated once, reused every step)
             srcs = (Q, scale, zero)
             if not pinned_out:
@@ -288,7 +296,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         torch.cuda.synchronize()
         if times is not None:
             for name, a, b in (("copy_in", 0, 1), ("hessian", 1, 2), ("init_rtn", 2, 3), ("cd_solve", 3, 4),
-                               ("loss_and_copy_out", 4, 5), ("total", 0, 5)):
+                               ("after_cd_solve", 4, 5), ("total", 0, 5)):
                 times.setdefault(name, []).append(ev[a].elapsed_time(ev[b]))
             times.setdefault("cd_kernel", []).append(stats["kernel_ms"])
             if want_cols:
@@ -373,6 +381,9 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
                **({"cd_kernel_ms_before_bcd": stats["cd_kernel_ms_before_bcd"], "loss_after_cd": stats["loss_after_cd"]}
                   if args.block == 2 else {})},
         "stages_ms": {k: mean(v) for k, v in times.items()},
+        # where the layer loss of the step comes from: inside cd_solve (half the dot product of the residual with the
+        # descent's final gradient) or after it (the product H E)
+        "loss_from": "descent gradient, inside cd_solve" if (args.block == 1 and not args.rows16) else "H E product, after cd_solve",
         "hessian": {"ms": hess_ms, "dense_equivalent_tflops": hess_flops / (hess_ms * 1e-3) / 1e12,
                     "executed_tflops": hess_exec / (hess_ms * 1e-3) / 1e12,
                     "executed_frac_of_bf16_sustained_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],

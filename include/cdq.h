@@ -215,6 +215,23 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
                               cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * cdq_cd_solve_steps followed by the loss of its result (paper: Eq. 1 with H = X^T X, the quantity
+ * Algorithm 1 descends on), sum_j e_j^T H e_j with e_j = W_hat[:, j] - W[:, j].  The descent keeps the
+ * gradient g_j = 2 H e_j of every column up to date, so the loss of the result is 1/2 sum_i e_ij g_ij:
+ * one dot product per column instead of the product H E.  FAST takes it that way on the shapes its
+ * register-resident kernels cover and agrees with cdq_layer_loss to ~1e-12 relative; VERIFY, and the
+ * remaining shapes, run cdq_layer_loss on the result.
+ *   loss     host pointer, may be NULL; the call synchronises when it is given.
+ *   per_col  [d_out] device doubles, may be NULL; not both NULL.
+ * Workspace: cdq_workspace_bytes(CDQ_CALL_CD_SOLVE, ...).
+ */
+cdq_status cdq_cd_solve_with_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                                  long long ldw, const cdq_grid_desc* grid, const float* scale,
+                                  const float* zero, unsigned char* Q, long long steps_per_col, cdq_mode mode,
+                                  cdq_cd_stats* stats, double* loss, double* per_col, void* ws, size_t ws_bytes,
+                                  void* stream);
+
+/*
  * Block coordinate descent with random blocks (paper: Algorithm 2; Algorithm 5 for sub-channel
  * grids), weight-unit form as above.  Step t cuts the d_in coordinates into d_in / block blocks
  * by a pseudo-random permutation pi (block u holds pi(block u), ..., pi(block u + block - 1)),

@@ -25,7 +25,7 @@ CALL_HESSIAN, CALL_INIT_RTN, CALL_CD_SOLVE, CALL_LAYER_LOSS, CALL_INIT_OWC_CD, C
 CALL_CD_SOLVE_ROWS16 = 6
 _MODES = {"fast": MODE_FAST, "verify": MODE_FP64_VERIFY, MODE_FAST: MODE_FAST, MODE_FP64_VERIFY: MODE_FP64_VERIFY}
 
-EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_cd_solve_rows16", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
+EXPORTS = ["cdq_hessian", "cdq_hessian_add_lambda", "cdq_init_rtn", "cdq_init_owc_cd", "cdq_cd_solve", "cdq_cd_solve_steps", "cdq_cd_solve_with_loss", "cdq_cd_solve_rows16", "cdq_bcd_solve", "cdq_layer_loss", "cdq_layer_loss_static",
            "cdq_workspace_bytes",
            "cdq_last_device_status", "cdq_last_error_detail", "cdq_status_string", "cdq_version",
            "cdq_kernel_launches", "cdq_debug_expire_wait", "cdq_debug_set_device_status"]
@@ -104,6 +104,9 @@ def load():
     lib.cdq_cd_solve_steps.restype = ci
     lib.cdq_cd_solve_steps.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ci, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_cd_solve_rows16.restype = ci
+    lib.cdq_cd_solve_with_loss.restype = ci
+    lib.cdq_cd_solve_with_loss.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ci, ctypes.POINTER(cdq_cd_stats),
+                                           ctypes.POINTER(ctypes.c_double), vp, vp, sz, vp]
     lib.cdq_cd_solve_rows16.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ll, ctypes.POINTER(cdq_cd_stats), vp, sz, vp]
     lib.cdq_layer_loss.restype = ci
     lib.cdq_layer_loss.argtypes = [vp, vp, ci, ll, ll, ll, gp, vp, vp, vp, ctypes.POINTER(ctypes.c_double), vp, ci, vp, sz, vp]
@@ -275,6 +278,37 @@ def cdq_cd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tens
             "loss_before": stats.loss_before, "loss_after": stats.loss_after, "kernel_ms": stats.kernel_ms}
 
 
+def cdq_cd_solve_with_loss(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,
+                           Q: torch.Tensor, steps_per_col: int, mode="fast", per_col: bool | torch.Tensor = False,
+                           ws: Workspace | None = None):
+    """Greedy coordinate descent (Q updated in place) and the loss of its result from the descent's own
+    gradient.  Returns (stats, loss) or (stats, loss, per_col)."""
+    _need_cuda(H, W, scale, zero, Q)
+    d_in, d_out = W.shape
+    assert H.shape == (d_in, d_in) and H.is_contiguous() and H.dtype == torch.float32
+    assert Q.shape == (d_in, d_out) and Q.is_contiguous() and Q.dtype == torch.uint8
+    assert scale.is_contiguous() and zero.is_contiguous() and W.stride(1) == 1
+    gd = grid.c()
+    stats = cdq_cd_stats()
+    loss = ctypes.c_double(0.0)
+    cols = None
+    if isinstance(per_col, torch.Tensor):
+        cols = per_col
+        assert cols.is_cuda and cols.dtype == torch.float64 and cols.is_contiguous() and cols.numel() == d_out
+    elif per_col:
+        cols = torch.empty(d_out, dtype=torch.float64, device=W.device)
+    ws = ws or _default_ws
+    wptr, wbytes = ws.get(workspace_bytes(CALL_CD_SOLVE, 0, d_in, d_out, grid, mode), W.device)
+    st = load().cdq_cd_solve_with_loss(H.data_ptr(), W.data_ptr(), _dtype_code(W), d_in, d_out, W.stride(0), ctypes.byref(gd),
+                                       scale.data_ptr(), zero.data_ptr(), Q.data_ptr(), int(steps_per_col), _MODES[mode],
+                                       ctypes.byref(stats), ctypes.byref(loss), cols.data_ptr() if cols is not None else None,
+                                       wptr, wbytes, _stream())
+    _check(st, "cdq_cd_solve_with_loss")
+    sd = {"steps": stats.steps, "committed": stats.committed, "columns_converged": stats.columns_converged,
+          "loss_before": stats.loss_before, "loss_after": stats.loss_after, "kernel_ms": stats.kernel_ms}
+    return (sd, loss.value, cols) if cols is not None else (sd, loss.value)
+
+
 def cdq_bcd_solve(H: torch.Tensor, W: torch.Tensor, grid: Grid, scale: torch.Tensor, zero: torch.Tensor,
                   Q: torch.Tensor, block: int, steps_per_col: int, seed: int = 0, mode="fast",
                   want_stats: bool = True, ws: Workspace | None = None):
@@ -369,11 +403,15 @@ def quantize_layer(X: torch.Tensor, W: torch.Tensor, grid: Grid, passes: int, la
         scale, zero, Q, gamma, _ = cdq_init_owc_cd(Wd, grid, H, mode=mode, ws=ws)
     else:
         scale, zero, Q, gamma = cdq_init_rtn(Wd, grid, H=H if grid.n_clip > 1 else None, mode=mode, ws=ws)
-    stats = cdq_cd_solve(H, Wd, grid, scale, zero, Q, passes, mode=mode, ws=ws, steps_per_col=steps_per_col)
-    out = {"H": H, "scale": scale, "zero": zero, "Q": Q, "gamma": gamma, "stats": stats}
+    budget = passes * Wd.shape[0] if steps_per_col is None else steps_per_col
     if bcd_steps > 0:
+        stats = cdq_cd_solve(H, Wd, grid, scale, zero, Q, passes, mode=mode, ws=ws, steps_per_col=steps_per_col)
+        out = {"H": H, "scale": scale, "zero": zero, "Q": Q, "gamma": gamma, "stats": stats}
         out["bcd_stats"] = cdq_bcd_solve(H, Wd, grid, scale, zero, Q, 2, bcd_steps, seed=seed, mode=mode, ws=ws)
-    out["loss"] = cdq_layer_loss(H, Wd, grid, scale, zero, Q, mode=mode, ws=ws)
+        out["loss"] = cdq_layer_loss(H, Wd, grid, scale, zero, Q, mode=mode, ws=ws)
+    else:   # the descent hands back the loss of its result
+        stats, loss = cdq_cd_solve_with_loss(H, Wd, grid, scale, zero, Q, budget, mode=mode, ws=ws)
+        out = {"H": H, "scale": scale, "zero": zero, "Q": Q, "gamma": gamma, "stats": stats, "loss": loss}
     if return_host:
         for k in ("scale", "zero", "Q"):
             out[k] = out[k].to("cpu", non_blocking=False)

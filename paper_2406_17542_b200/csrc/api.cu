@@ -345,7 +345,8 @@ cdq_status cdq_init_owc_cd(const void* W, cdq_dtype wt, long long d_in, long lon
 static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,
                                 const cdq_grid_desc* grid, const float* scale, const float* zero, unsigned char* Q,
                                 long long steps_per_col, int block, unsigned long long seed, cdq_mode mode,
-                                cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream, bool rows16 = false) {
+                                cdq_cd_stats* stats, void* ws, size_t ws_bytes, void* stream, bool rows16 = false,
+                                double* loss_out = nullptr, double* per_col_out = nullptr) {
   if (!H || !W || !scale || !zero || !Q || !valid_dtype(wt) || !valid_mode(mode) || steps_per_col < 0)
     return CDQ_ERR_INVALID_ARG;
   if (!aligned16(H)) return CDQ_ERR_INVALID_ARG;
@@ -418,6 +419,20 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
   }
   if (stats) CDQ_CUDA(cudaEventRecord(ev1, st));
   CDQ_CUDA(launch_transpose_u8(Qt, d_out, d_in, L.ldg, Q, d_out, st));
+  const bool want_loss = loss_out || per_col_out;
+  // The register-resident kernels leave the gradient of their result in G: the loss is then a dot product
+  // per column.  The other kernels' results get the loss from its definition.
+  const bool loss_from_g = want_loss && fast_cd && block == 1 && !rows16;
+  if (loss_from_g) {
+    double* col_after = per_col_out ? per_col_out : col_loss;   // col_loss has been summed into loss_sum[0] by now
+    CDQ_CUDA(launch_residual_f64(codes_src(ly, Q), d_in, E, st));
+    CDQ_CUDA(launch_loss_from_gradient(E, G, L.ldg, d_in, d_out, col_after, st));
+    if (loss_out) {
+      CDQ_CUDA(launch_sum_f64_tree(col_after, d_out, loss_sum + 1, st));
+      CDQ_CUDA(cudaMemcpyAsync(loss_out, loss_sum + 1, sizeof(double), cudaMemcpyDeviceToHost, st));
+      if (!stats) CDQ_CUDA(cudaStreamSynchronize(st));
+    }
+  }
   if (stats) {
     CdCounters hc;
     double lb = 0.0;
@@ -432,8 +447,11 @@ static cdq_status cd_solve_impl(const float* H, const void* W, cdq_dtype wt, lon
     float ms = 0.f;
     CDQ_CUDA(cudaEventElapsedTime(&ms, ev0, ev1));
     stats->kernel_ms = (double)ms;
-    return read_device_status_after_sync();
+    const cdq_status ds = read_device_status_after_sync();
+    if (ds != CDQ_OK) return ds;
   }
+  if (want_loss && !loss_from_g)
+    return cdq_layer_loss(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, loss_out, per_col_out, mode, ws, ws_bytes, stream);
   return CDQ_OK;
 }
 
@@ -451,6 +469,15 @@ cdq_status cdq_cd_solve_steps(const float* H, const void* W, cdq_dtype wt, long 
                               size_t ws_bytes, void* stream) {
   return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, 1, 0ull, mode, stats, ws,
                        ws_bytes, stream);
+}
+
+cdq_status cdq_cd_solve_with_loss(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,
+                                  long long ldw, const cdq_grid_desc* grid, const float* scale, const float* zero,
+                                  unsigned char* Q, long long steps_per_col, cdq_mode mode, cdq_cd_stats* stats,
+                                  double* loss, double* per_col, void* ws, size_t ws_bytes, void* stream) {
+  if (!loss && !per_col) return CDQ_ERR_INVALID_ARG;
+  return cd_solve_impl(H, W, wt, d_in, d_out, ldw, grid, scale, zero, Q, steps_per_col, 1, 0ull, mode, stats, ws,
+                       ws_bytes, stream, false, loss, per_col);
 }
 
 cdq_status cdq_cd_solve_rows16(const float* H, const void* W, cdq_dtype wt, long long d_in, long long d_out,

@@ -64,6 +64,46 @@ cudaError_t launch_transpose_u8(const unsigned char* src, long long rows, long l
   return cudaGetLastError();
 }
 
+// col_loss[j] = 1/2 sum_i E[i][j] G[j][i]: with g = 2 H e the loss e^T H e (Eq. 1) of a column is half the dot
+// product of its residual and its gradient.  One CTA per 32 columns, rows in ascending tiles of 32, every column's
+// sum kept by one warp: the result does not depend on the launch shape.
+__global__ void __launch_bounds__(256) loss_from_gradient_kernel(const double* __restrict__ E, const double* __restrict__ G,
+                                                                 long long ldg, long long d_in, long long d_out,
+                                                                 double* __restrict__ col_loss) {
+  __shared__ double tile[32][33];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const long long j0 = (long long)blockIdx.x * 32;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (long long i0 = 0; i0 < d_in; i0 += 32) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {   // E[i0 + ty + 8 r][j0 + tx], contiguous along the columns
+      const long long i = i0 + ty + 8 * r, j = j0 + tx;
+      tile[ty + 8 * r][tx] = (i < d_in && j < d_out) ? E[i * d_out + j] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {   // G[j0 + ty + 8 r][i0 + tx], contiguous along the rows
+      const long long i = i0 + tx, j = j0 + ty + 8 * r;
+      if (i < d_in && j < d_out) acc[r] += tile[tx][ty + 8 * r] * G[j * ldg + i];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    double v = acc[r];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const long long j = j0 + ty + 8 * r;
+    if (tx == 0 && j < d_out) col_loss[j] = 0.5 * v;
+  }
+}
+
+cudaError_t launch_loss_from_gradient(const double* E, const double* G, long long ldg, long long d_in, long long d_out,
+                                      double* col_loss, cudaStream_t st) {
+  { loss_from_gradient_kernel<<<(unsigned)((d_out + 31) / 32), 256, 0, st>>>(E, G, ldg, d_in, d_out, col_loss); count_launch(); }
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float4 ld_row4(const float* p) {
   float4 v;
@@ -245,13 +285,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_fast_kernel(CdParams p) {
       my_dsum += SMODE == kPerChannel ? col_dsum * ((double)a_col * (double)a_col) : col_dsum;
     }
 
-    // ---- write the codes back ----
+    // ---- write the codes back, and the gradient of the result (weight units) ----
     {
       unsigned char* qcol = p.Qt + j * p.ldq;
+      double* gcol = p.G + j * p.ldg;
+      const double ga = SMODE == kPerChannel ? (double)a_col : 1.0;
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         const int chunk = tid + NT * k;
-        if (EXACT || chunk < nchunks) *reinterpret_cast<unsigned*>(qcol + (long long)chunk * 4) = qp[k];
+        if (EXACT || chunk < nchunks) {
+          *reinterpret_cast<unsigned*>(qcol + (long long)chunk * 4) = qp[k];
+          *reinterpret_cast<double2*>(gcol + (long long)chunk * 4) = make_double2(g[4 * k] * ga, g[4 * k + 1] * ga);
+          *reinterpret_cast<double2*>(gcol + (long long)chunk * 4 + 2) = make_double2(g[4 * k + 2] * ga, g[4 * k + 3] * ga);
+        }
       }
     }
   }

@@ -240,13 +240,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       my_dsum += SMODE == kPerChannel ? col_dsum * ((double)a_col * (double)a_col) : col_dsum;
     }
 
-    // ---- write the codes back ----
+    // ---- write the codes back, and the gradient of the result (weight units) ----
     if (!frozen) {
       unsigned char* qcol = p.Qt + j * p.ldq;
+      double* gcol = p.G + j * p.ldg;
+      const double ga = SMODE == kPerChannel ? (double)a_col : 1.0;
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         const int cs = tid + NT * k;
-        if (exact || cs < nchs) *reinterpret_cast<unsigned*>(qcol + (long long)cs * 4) = qp[k];
+        if (exact || cs < nchs) {
+          *reinterpret_cast<unsigned*>(qcol + (long long)cs * 4) = qp[k];
+          *reinterpret_cast<double2*>(gcol + (long long)cs * 4) = make_double2(g[4 * k] * ga, g[4 * k + 1] * ga);
+          *reinterpret_cast<double2*>(gcol + (long long)cs * 4 + 2) = make_double2(g[4 * k + 2] * ga, g[4 * k + 3] * ga);
+        }
       }
     }
   }

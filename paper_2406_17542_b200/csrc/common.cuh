@@ -124,6 +124,9 @@ long long cd_fast_pad(long long d_in);      // padded length of hdiag / hs
 bool cd_fast_supported(long long d_in, long long g);
 // hdiag = H_ii, hs = 0.5 / H_ii
 cudaError_t launch_diag(const float* H, long long d_in, long long d_pad, float* hdiag, float* hs, cudaStream_t st);
+// col_loss[j] = 1/2 sum_i E[i][j] G[j][i] (E [d_in, d_out], G [d_out, ldg]): e^T H e from the gradient g = 2 H e.
+cudaError_t launch_loss_from_gradient(const double* E, const double* G, long long ldg, long long d_in, long long d_out,
+                                      double* col_loss, cudaStream_t st);
 // H16 (may be NULL): bf16 copy of H for the rows of the update; cudaErrorNotSupported if the shape has no such kernel
 cudaError_t launch_cd_fast(const Layer& ly, const __nv_bfloat16* H16, double* G, long long ldg, unsigned char* Qt,
                            long long ldq, const float* hdiag, const float* hs, long long steps_per_col,
