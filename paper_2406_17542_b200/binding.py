@@ -416,3 +416,54 @@ def quantize_layer(X: torch.Tensor, W: torch.Tensor, grid: Grid, passes: int, la
         for k in ("scale", "zero", "Q"):
             out[k] = out[k].to("cpu", non_blocking=False)
     return out
+
+
+_copy_streams: dict = {}
+
+
+def quantize_layers(layers, grid: Grid, passes: int, device="cuda:0", ws: Workspace | None = None,
+                    host_buffers: dict | None = None, **kw):
+    """Generator over an iterable of (X, W) pairs held in (pinned) host memory: yields quantize_layer's result for
+    every layer in turn, with codes, scales and zeros back in pinned host buffers.
+
+    The inputs of layer k + 1 are uploaded on a second stream while layer k computes (two input buffers on the
+    device), so that from the second layer on the host-to-device copy costs nothing unless it is longer than
+    the layer's compute.  The host buffers of a result are reused by the next layer of the same shape: copy what
+    must outlive the next iteration (host_buffers: a dict that keeps them across calls).  Keyword arguments are
+    quantize_layer's (lambda_rel, mode, init, ...)."""
+    dev = torch.device(device)
+    if dev not in _copy_streams:
+        _copy_streams[dev] = torch.cuda.Stream(dev)
+    copy_stream = _copy_streams[dev]
+    main = torch.cuda.current_stream(dev)
+    host_out: dict = host_buffers if host_buffers is not None else {}
+    it = iter(layers)
+
+    def upload(pair):
+        X, W = pair
+        with torch.cuda.stream(copy_stream):
+            Xd = X.to(dev, non_blocking=True)
+            Wd = W.to(dev, non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(copy_stream)
+        return Xd, Wd, ev
+
+    nxt = next(it, None)
+    pending = upload(nxt) if nxt is not None else None
+    while pending is not None:
+        Xd, Wd, ev = pending
+        nxt = next(it, None)
+        pending = upload(nxt) if nxt is not None else None   # in flight while this layer computes
+        main.wait_event(ev)
+        out = quantize_layer(Xd, Wd, grid, passes, device=device, ws=ws, return_host=False, **kw)
+        Xd.record_stream(main)
+        Wd.record_stream(main)
+        for k in ("scale", "zero", "Q"):
+            t = out[k]
+            key = (k, tuple(t.shape), t.dtype)
+            if key not in host_out:
+                host_out[key] = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+            host_out[key].copy_(t, non_blocking=True)
+            out[k] = host_out[key]
+        main.synchronize()
+        yield out
