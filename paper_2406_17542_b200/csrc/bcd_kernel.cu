@@ -550,7 +550,7 @@ static cudaError_t launch_bcd_cfg(const CdParams& p, const uint4* tab, int nt, c
   const int g_in_smem = !force_global && smem + sizeof(double) * (size_t)p.ldg <= budget ? 1 : 0;
   if (g_in_smem) smem += sizeof(double) * (size_t)p.ldg;
   cudaError_t e;
-  if (smem > 48 * 1024) {
+  if (smem > 32 * 1024) {   // the 48 KB that need no opt-in include the kernel's static shared memory
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }

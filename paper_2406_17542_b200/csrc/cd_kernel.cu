@@ -323,7 +323,7 @@ static cudaError_t launch_cd_cfg(CdParams p, int nt, cudaStream_t st) {
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const size_t smem = SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count;
   cudaError_t e;
-  if (smem > 48 * 1024) {
+  if (smem > 32 * 1024) {   // the 48 KB that need no opt-in include the kernel's static shared memory
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }

@@ -3,12 +3,11 @@
 // aligned (d_in % 4 == 0).
 //
 // Same step as cd_kernel.cu -- score, argmin, read row i*, update the gradient -- but the row
-// H[i*, :] is fetched by bulk asynchronous copies (cp.async.bulk, no multicast) into shared
-// memory, one copy and one mbarrier per chunk slot of the team (or one for the whole row, see PS),
-// each issued by a single thread.
+// H[i*, :] is fetched by one bulk asynchronous copy (cp.async.bulk, no multicast) into shared
+// memory, issued by a single thread and completed on one mbarrier.
 // The copy engine keeps the whole row in flight at once (loads issued by the threads themselves
-// did not: the SM tracks only so many outstanding misses), the sweep starts on the first piece
-// while the others are still landing, and the row no longer occupies 32 registers per thread.
+// did not: the SM tracks only so many outstanding misses), and the row no longer occupies
+// registers.
 //
 // Waits on the copy barriers are bounded by a cycle count.  A thread whose wait runs out enters the
 // argmin with a key that no real move can have; the whole team sees it after the exchange, starts no
@@ -30,11 +29,7 @@ constexpr unsigned kAbortKey = 0u;    // below the key of every real move (a mov
 template <int NCH, int MAXNT, int MINB, int SMODE, bool ROW16>
 __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
-  // chunk slots per bulk copy: one copy for the whole row, except for the 768 x 6 team of the longest
-  // rows (74 KB), which is quicker with one copy per slot
-  constexpr int PS = (NCH == 4 && MAXNT == 896) ? 4 : ((NCH == 8 && MAXNT == 256) ? 8 : ((NCH == 4 && MAXNT == 256) ? 4 : 1));
-  constexpr int NP = NCH / PS;                              // bulk copies per row
-  __shared__ __align__(8) unsigned long long s_bar[NP];
+  __shared__ __align__(8) unsigned long long s_bar;   // completion of the row's copy
   __shared__ __align__(8) uint2 s_exch[2][32];
   __shared__ int s_col;
 
@@ -64,15 +59,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   // slots past the end of the row stay zero: no copy ever writes there
   for (int t = tid; t < NCH * NT * CHB / 8; t += NT) reinterpret_cast<uint2*>(row_s)[t] = make_uint2(0u, 0u);
   if (tid == 0) {
-#pragma unroll
-    for (int k = 0; k < NP; ++k) mbar_init(smem_u32(&s_bar[k]), 1);
+    mbar_init(smem_u32(&s_bar), 1);
     mbar_fence_init();
   }
-  // bytes of the row piece behind chunk slot k (0 when the slot lies past the row)
-  auto piece_bytes = [&](int k) -> uint32_t {
-    const int lo = NT * PS * k, hi = min(NT * PS * (k + 1), nchs);
-    return hi > lo ? (uint32_t)(hi - lo) * (uint32_t)CHB : 0u;
-  };
+  const uint32_t row_bytes = (uint32_t)nchs * (uint32_t)CHB;
   __syncthreads();
   fence_proxy_async_smem();  // zero fill before the first copy lands
 
@@ -131,21 +121,15 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
     double c2 = 0.0;       // twice the step being applied (code units when per-channel)
     double col_dsum = 0.0;
     bool done = frozen;
-    // Requests row `off / d_in` of H: piece k by the first lane of warp k (by thread 0 when the team has fewer warps).
-    // Called when every thread is past its reads of the previous row (behind the barrier of the argmin, or of the
-    // column prologue), and as early as the row is known: what follows the argmin overlaps with the copy.
+    // Requests row `off / d_in` of H.  Called when every thread is past its reads of the previous row (behind the
+    // barrier of the argmin, or of the column prologue), and as early as the row is known: what follows the argmin
+    // overlaps with the copy.
     auto request_row = [&](long long off) {
-      const unsigned char* src = ROW16 ? reinterpret_cast<const unsigned char*>(p.H16 + off)
-                                       : reinterpret_cast<const unsigned char*>(p.H + off);
-#pragma unroll
-      for (int k = 0; k < NP; ++k) {
-        const bool issuer = nwarps >= NP ? (warp == k && lane == 0) : tid == 0;
-        const uint32_t bytes = piece_bytes(k);
-        if (issuer && bytes) {
-          const uint32_t bar = smem_u32(&s_bar[k]);
-          mbar_expect_tx(bar, bytes);
-          bulk_load(smem_u32(row_s + (size_t)NT * PS * k * CHB), src + (size_t)NT * PS * k * CHB, bytes, bar);
-        }
+      if (tid == 0) {
+        const unsigned char* src = ROW16 ? reinterpret_cast<const unsigned char*>(p.H16 + off)
+                                         : reinterpret_cast<const unsigned char*>(p.H + off);
+        mbar_expect_tx(smem_u32(&s_bar), row_bytes);
+        bulk_load(smem_u32(row_s), src, row_bytes, smem_u32(&s_bar));
       }
     };
     if (!done) request_row(0);
@@ -160,9 +144,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
         const float4 hs = __ldg(reinterpret_cast<const float4*>(p.hs) + cs);
         float a, ia;
         chunk_scale(k, a, ia);
-        if ((k % PS) == 0 && (exact || NT * k < nchs)) {
-          if (!mbar_wait_clock32(smem_u32(&s_bar[k / PS]), phase, kWaitCycles)) timed_out = true;
-        }
+        if (k == 0 && !mbar_wait_clock32(smem_u32(&s_bar), phase, kWaitCycles)) timed_out = true;
         float4 rv;
         if constexpr (ROW16) {
           const uint2 rr = reinterpret_cast<const uint2*>(row_s)[cs];
@@ -203,9 +185,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
       }
       if (m == kAbortKey) {   // a copy never landed: wait (bounded) for the pieces of this row, then give up
         if (tid == 0) {
-#pragma unroll
-          for (int k = 0; k < NP; ++k)
-            if (piece_bytes(k)) mbar_wait_clock32(smem_u32(&s_bar[k]), phase ^ 1u, kWaitCycles);
+          mbar_wait_clock32(smem_u32(&s_bar), phase ^ 1u, kWaitCycles);
           atomicCAS(p.status, (int)kFlagOk, (int)kFlagWaitTimeout);
         }
         aborted = true;
@@ -277,7 +257,7 @@ cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const size_t smem = (size_t)NCH * nt * (ROW16 ? 8 : 16) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
   cudaError_t e;
-  if (smem > 48 * 1024) {
+  if (smem > 32 * 1024) {   // the 48 KB that need no opt-in include the kernel's static shared memory
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
@@ -314,11 +294,23 @@ cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st) {
   if (p.H16 && ((p.d_in & 7) != 0 || (reinterpret_cast<uintptr_t>(p.H16) & 15) != 0)) return cudaErrorNotSupported;
   const long long ch = p.d_in >> 2;
   auto team = [&](long long chunks, int nch) { return (int)((chunks + nch - 1) / nch + 31) / 32 * 32; };
-  if (ch <= 128) return launch_mode<2, 64, 8>(p, team(ch, 2), st);
-  if (ch <= 1024) return launch_mode<4, 256, 3>(p, team(ch, 4), st);
+  // (called for rows of more than 2048 entries)  Rows up to 8192 entries: several teams per SM.
+  if (ch <= 1024) return launch_mode<8, 128, 4>(p, team(ch, 8), st);
   if (ch <= 2048) return launch_mode<8, 256, 2>(p, team(ch, 8), st);
-  if (ch <= 3584) return launch_mode<4, 896, 1>(p, team(ch, 4), st);
-  if (ch <= 4608) return launch_mode<6, 768, 1>(p, team(ch, 6), st);
+  // Longer rows: one team per SM.  Few threads with many chunks each beat many threads with few (no spills,
+  // a cheaper argmin exchange, fixed costs per thread spread over more state), and a team of 12 or 16 full
+  // warps beats a ragged one, so the shape is the smallest of 5..8 x 512 and 7..12 x 384 chunk slots that
+  // holds the row.  Cycles per move and SM, against the 4 x 896 / 6 x 768 teams used before: d_in 10240 4526
+  // (4813), 11008 4752 (5079), 14336 5484 (5903), 15360 5865 (7482), 16384 6172 (8022), 18432 6921 (8418).
+  if (ch <= 2560) return launch_mode<5, 512, 1>(p, team(ch, 5), st);
+  if (ch <= 2688) return launch_mode<7, 384, 1>(p, team(ch, 7), st);
+  if (ch <= 3072) return launch_mode<6, 512, 1>(p, team(ch, 6), st);
+  if (ch <= 3456) return launch_mode<9, 384, 1>(p, team(ch, 9), st);
+  if (ch <= 3584) return launch_mode<7, 512, 1>(p, team(ch, 7), st);
+  if (ch <= 3840) return launch_mode<10, 384, 1>(p, team(ch, 10), st);
+  if (ch <= 4096) return launch_mode<8, 512, 1>(p, team(ch, 8), st);
+  if (ch <= 4224) return launch_mode<11, 384, 1>(p, team(ch, 11), st);
+  if (ch <= 4608) return launch_mode<12, 384, 1>(p, team(ch, 12), st);
   return cudaErrorNotSupported;
 }
 

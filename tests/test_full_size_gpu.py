@@ -134,6 +134,13 @@ def test_mid_size_columns_sampled():
     _run(inputs.CONFIGS["C3"].scaled(d_in=6144, d_out=296, seed=61), rows=8192, n_sample=32)
 
 
+def test_rows_of_exactly_48_kb_sampled():
+    """d_in = 12288 per-channel: the row takes exactly 48 KB of dynamic shared memory, which together with the
+    kernel's static shared memory needs the opt-in for large shared memory (a launch error before it was
+    requested for this size too)."""
+    _run(inputs.CONFIGS["C3"].scaled(d_in=12288, d_out=148, seed=63), rows=8192, n_sample=16)
+
+
 def test_ragged_long_columns_sampled():
     """d_in = 11008 (not a multiple of the team's footprint: the last chunk slots reach past the row), rows
     from HBM by one bulk copy, 296 columns, the oracle on 32 of them."""
@@ -144,3 +151,34 @@ def test_long_columns_whose_length_is_not_a_multiple_of_four_sampled():
     """d_in = 6146 (rows of H are then not 16-byte aligned: no bulk copies, the kernel that keeps the row in
     registers runs with scalar loads at the ragged end), 148 columns, the oracle on 32 of them."""
     _run(inputs.CONFIGS["C3"].scaled(d_in=6146, d_out=148, seed=71), rows=8192, n_sample=32)
+
+
+# Row lengths (in entries) at which the kernel that stages rows through shared memory changes its team shape,
+# each with a length just inside the next shape; 12224 and 12288 are the lengths whose row fills the 48 KB of
+# shared memory that need no opt-in (together with the kernel's own static shared memory they exceed it).
+_SHAPE_EDGES = [4 * c for c in (1024, 2048, 2560, 2688, 3072, 3456, 3584, 3840, 4096, 4224, 4608)]
+ROW_LENGTHS = {
+    0: sorted(set([2304, 12224] + _SHAPE_EDGES + [d + 16 for d in _SHAPE_EDGES[:-1]])),
+    128: sorted(set([2304, 12160] + _SHAPE_EDGES + [d + 128 for d in _SHAPE_EDGES[:-1]])),
+}
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_every_team_shape_of_the_long_row_kernel(group):
+    """Every team shape of the long-row descent kernel, with a full and with a ragged team: 6 columns, 24 steps
+    each, the loss of the result from the descent's gradient; codes, grids and losses against the oracle."""
+    dev = "cuda:0"
+    for d_in in ROW_LENGTHS[group]:
+        cfg = inputs.CONFIGS["C3"].scaled(d_in=d_in, d_out=6, bits=3, group_size=group, n_clip=1, clip_lo=1.0, clip_hi=1.0,
+                                          seed=500 + d_in % 97)
+        Hd = _h_from_rows(cfg, 512, ridge=1e-2)
+        Wd = inputs.make_w(cfg, device=dev)
+        g = grid_of(cfg)
+        scale, zero, Q0, gamma = B.cdq_init_rtn(Wd, g)
+        Q = Q0.clone()
+        budget = 24
+        stats, loss, per = B.cdq_cd_solve_with_loss(Hd, Wd, g, scale, zero, Q, budget, per_col=True)
+        assert B.load().cdq_last_device_status() == 0
+        assert stats["committed"] == budget * cfg.d_out, (d_in, stats)
+        compare_with_oracle(cfg, Hd.cpu().numpy(), Hd, Wd, np.arange(cfg.d_out), g, scale, zero, Q0, Q, gamma, per, budget,
+                            label=f"d_in={d_in} g={group}")
