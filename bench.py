@@ -43,14 +43,14 @@ L2_BYTES = 126e6
 # capture divided by the moves of that capture), keyed by (kernel, d_in); a kernel and shape without a
 # capture of the kernel as it stands reports traffic null.  Each entry names the summary it comes from.
 NCU_TRAFFIC_PER_MOVE: dict = {
-    ("cd_tma_kernel", 14336): (44577.0, "profiles/cd_tma_kernel_C3_592cols.md"),
+    ("cd_tma_kernel", 14336): (44549.0, "profiles/cd_tma_kernel_C3_592cols.md"),
 }
 
 
 def descent_kernel_name(cfg, block: int) -> str:
     if block == 2:
         return "bcd2_kernel"
-    return "cd_tma_kernel" if cfg.d_in > 2048 and cfg.d_in % 4 == 0 else "cd_fast_kernel"
+    return "cd_tma_kernel" if cfg.d_in > 1536 and cfg.d_in % 4 == 0 else "cd_fast_kernel"
 
 
 def load_peaks():

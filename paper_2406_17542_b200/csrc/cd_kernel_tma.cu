@@ -294,7 +294,7 @@ cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st) {
   if (p.H16 && ((p.d_in & 7) != 0 || (reinterpret_cast<uintptr_t>(p.H16) & 15) != 0)) return cudaErrorNotSupported;
   const long long ch = p.d_in >> 2;
   auto team = [&](long long chunks, int nch) { return (int)((chunks + nch - 1) / nch + 31) / 32 * 32; };
-  // (called for rows of more than 2048 entries)  Rows up to 8192 entries: several teams per SM.
+  // (called for rows of more than 1536 entries)  Rows up to 8192 entries: several teams per SM.
   if (ch <= 1024) return launch_mode<8, 128, 4>(p, team(ch, 8), st);
   if (ch <= 2048) return launch_mode<8, 256, 2>(p, team(ch, 8), st);
   // Longer rows: one team per SM.  Few threads with many chunks each beat many threads with few (no spills,
