@@ -301,6 +301,18 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
             times.setdefault("cd_kernel", []).append(stats["kernel_ms"])
             if want_cols:
                 keep.update(H=H, W=Wd, scale=scale, zero=zero, Q0=Q0, Q=Q, gamma=gamma, per=per)
+        if last and not host:
+            # outside the step: the stand-alone loss call (the product H E on the result) for the record, and how far
+            # the step's own loss is from it
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n0 = lib.cdq_kernel_launches()
+            t0.record()
+            ref_loss = B.cdq_layer_loss(H, Wd, grid, scale, zero, Q, ws=ws)
+            t1.record()
+            torch.cuda.synchronize()
+            keep["untimed_launches"] = lib.cdq_kernel_launches() - n0
+            keep["layer_loss_call"] = {"ms": t0.elapsed_time(t1), "loss": ref_loss,
+                                       "step_loss_rel_diff": abs(loss - ref_loss) / abs(ref_loss) if ref_loss else 0.0}
         return stats, loss, d2h
 
     def timed(host: bool):
@@ -315,7 +327,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
             flush.fill_(1)           # evict L2 between timed iterations (not timed)
             torch.cuda.synchronize()
             stats, loss, d2h = one_step(host, times, last=it == steps - 1)
-        launches = lib.cdq_kernel_launches() - launches0
+        launches = lib.cdq_kernel_launches() - launches0 - keep.pop("untimed_launches", 0)
         multi.barrier(world)
         return times, stats, loss, d2h, launches
 
@@ -410,6 +422,7 @@ def run_config(B, cfg, args, steps: int, warmup: int, dev, world: int, rank: int
         # where the layer loss of the step comes from: inside cd_solve (half the dot product of the residual with the
         # descent's final gradient) or after it (the product H E)
         "loss_from": "descent gradient, inside cd_solve" if (args.block == 1 and not args.rows16) else "H E product, after cd_solve",
+        "layer_loss_call": keep.get("layer_loss_call"),
         "hessian": {"ms": hess_ms, "dense_equivalent_tflops": hess_flops / (hess_ms * 1e-3) / 1e12,
                     "executed_tflops": hess_exec / (hess_ms * 1e-3) / 1e12,
                     "executed_frac_of_bf16_sustained_peak": hess_exec / (hess_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
@@ -522,6 +535,7 @@ def main():
                                 if args.shard else "one independent layer per GPU, no collective")},
         "sec_per_layer": rec["sec_per_layer"], "cd": rec["cd"], "stages_ms": rec["stages_ms"], "hessian": rec["hessian"],
         "roofline": rec["roofline"], "e2e": rec["e2e"], "gpu_launches": rec["gpu_launches"], "clocks": rec["clocks"],
+        "loss_from": rec["loss_from"], "layer_loss_call": rec["layer_loss_call"],
     }
     if "parity" in rec:
         out["parity"] = rec["parity"]
