@@ -566,7 +566,9 @@ def main():
 
 def run_reference(args, cfg, workload):
     """The oracle as the timed program: each step is one bounded sample of the workload, sized from a short probe
-    so that a step stays near five seconds (about half Hessian, half grid + descent + loss) whatever d_in is."""
+    so that the whole run (warm-up and timed steps) takes about two and a half minutes whatever d_in and the step
+    counts are: a step gets 150 s / (steps + warmup), at least 2 s and at most 20 s, half of it for the Hessian rows
+    and half for grid + descent + loss of the sampled columns."""
     import oracle
     probe_rows, probe_cols = 64, 2
     X, W = inputs.make_layer(cfg.scaled(n=min(cfg.n, 8192), d_out=min(cfg.d_out, 256)), device="cpu")
@@ -580,8 +582,9 @@ def run_reference(args, cfg, workload):
                     cfg.group_size)
     # columns run in parallel over the host threads: one thread's rate times the threads is what more columns get
     cols_per_s = probe_cols / max(time.perf_counter() - t0, 1e-6) * max(oracle.num_threads() // 2, 1)
-    n_rows = int(min(X.shape[0], max(probe_rows, rows_per_s * 2.5)))
-    n_cols = int(min(W.shape[1], max(probe_cols, cols_per_s * 2.5)))
+    step_s = min(20.0, max(2.0, 150.0 / max(args.steps + max(args.warmup, 0), 1)))
+    n_rows = int(min(X.shape[0], max(probe_rows, rows_per_s * step_s / 2)))
+    n_cols = int(min(W.shape[1], max(probe_cols, cols_per_s * step_s / 2)))
     for _ in range(max(args.warmup, 0)):
         run_oracle_sample(cfg, X, W, n_rows, n_cols)
     vals, secs = [], []
@@ -597,7 +600,7 @@ def run_reference(args, cfg, workload):
         "config": {"workload": workload, "l2": "not applicable (host cores)",
                    "per_rank": "rank 0 only: the CPU oracle on a bounded sample per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": r["cores"], "kind": "oracle",
-                         "sample": r["sample"] + " (sample sized from a probe so that a step takes about five seconds)"},
+                         "sample": r["sample"] + f" (sample sized from a probe for about {step_s:.0f} s per step)"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
