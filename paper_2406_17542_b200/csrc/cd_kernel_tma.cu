@@ -40,8 +40,14 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
   const float top = kMagic + (float)p.L;
 
   constexpr int CHB = ROW16 ? 8 : 16;                                   // bytes of a chunk of 4 row entries
+  // H_ii and 0.5 / H_ii of the team's chunk slots sit in shared memory too: they are the same for every column and
+  // every sweep reads them (8 d_in bytes); from L1 they cost more latency, and beside the row buffer of the longest
+  // rows the L1 does not hold them.  (148 to 1184 columns, before -> after: 2048 entries 12.4 -> 10.6 ms, 6144
+  // 23.4 -> 19.4, 8192 42.1 -> 36.8, 14336 163.7 -> 160.1, 18432 67.5 -> 60.4.)
   unsigned char* row_s = dyn_smem;                                      // [NCH * NT] chunks
-  float2* ag_s = reinterpret_cast<float2*>(row_s + (size_t)NCH * NT * CHB);  // [ag_count] (a, 1/a), grouped modes
+  float4* hd_s = reinterpret_cast<float4*>(row_s + (size_t)NCH * NT * CHB);   // [NCH * NT] H_ii
+  float4* hs_s = hd_s + NCH * NT;                                             // [NCH * NT] 0.5 / H_ii
+  float2* ag_s = reinterpret_cast<float2*>(hs_s + NCH * NT);                  // [ag_count] (a, 1/a), grouped modes
   auto group_of = [&](unsigned i) -> unsigned { return p.g == 1 ? i : __umulhi(i, p.gmagic); };
   const int g4 = SMODE == kGroupFast ? (int)(p.g >> 2) : 1;
   const float2* ag_mine = ag_s + (SMODE == kGroupFast ? tid / g4 : 0);
@@ -58,6 +64,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
 
   // slots past the end of the row stay zero: no copy ever writes there
   for (int t = tid; t < NCH * NT * CHB / 8; t += NT) reinterpret_cast<uint2*>(row_s)[t] = make_uint2(0u, 0u);
+  for (int t = tid; t < NCH * NT; t += NT) {   // (the arrays are padded past every team's footprint)
+    hd_s[t] = __ldg(reinterpret_cast<const float4*>(p.hdiag) + t);
+    hs_s[t] = __ldg(reinterpret_cast<const float4*>(p.hs) + t);
+  }
   if (tid == 0) {
     mbar_init(smem_u32(&s_bar), 1);
     mbar_fence_init();
@@ -140,8 +150,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) cd_tma_kernel(CdParams p) {
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         const int cs = tid + NT * k;
-        const float4 hd = __ldg(reinterpret_cast<const float4*>(p.hdiag) + cs);
-        const float4 hs = __ldg(reinterpret_cast<const float4*>(p.hs) + cs);
+        const float4 hd = hd_s[cs];
+        const float4 hs = hs_s[cs];
         float a, ia;
         chunk_scale(k, a, ia);
         if (k == 0 && !mbar_wait_clock32(smem_u32(&s_bar), phase, kWaitCycles)) timed_out = true;
@@ -255,7 +265,8 @@ cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const size_t smem = (size_t)NCH * nt * (ROW16 ? 8 : 16) + (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
+  const size_t smem = (size_t)NCH * nt * (ROW16 ? 8 : 16) + (size_t)NCH * nt * 32 +
+                      (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
   cudaError_t e;
   if (smem > 32 * 1024) {   // the 48 KB that need no opt-in include the kernel's static shared memory
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
