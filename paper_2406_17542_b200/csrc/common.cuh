@@ -81,6 +81,8 @@ struct ResidualSrc {
   long long g, d_out;      // d_out: columns of the layer (the width of W's companions scale, zero, Q, mn, mx)
   const int* col_idx;      // NULL: E has a column for every layer column; else E column c is layer column col_idx[c] ...
   long long n_cols;        // ... and E is [d_in, n_cols]
+  const int* col_gamma;    // OWC path, with col_idx: E column c takes the clipping strength gammas[col_gamma[c]] ...
+  const double* gammas;    // ... instead of `gamma` (NULL: `gamma` for every column)
 };
 cudaError_t launch_residual_f64(const ResidualSrc& src, long long d_in, double* E, cudaStream_t st);
 

@@ -94,7 +94,8 @@ __global__ void residual_kernel(ResidualSrc s, long long d_in, double* __restric
   double a, b, q;
   if (s.use_gamma) {
     const double lo = (double)s.mn[t * s.d_out + j], hi = (double)s.mx[t * s.d_out + j];
-    const float a32 = (float)__ddiv_rn(__dmul_rn(s.gamma, __dadd_rn(hi, -lo)), (double)s.L);
+    const double gamma = s.col_gamma ? s.gammas[s.col_gamma[c]] : s.gamma;
+    const float a32 = (float)__ddiv_rn(__dmul_rn(gamma, __dadd_rn(hi, -lo)), (double)s.L);
     a = (double)a32;
     b = lo;
     q = 0.0;
@@ -159,8 +160,7 @@ __global__ void owc_candidates_kernel(const double* __restrict__ screen, int n_c
   }
 }
 
-// One CTA per clipping strength: its candidate columns in ascending order, padded by repeating the last one to a
-// multiple of 128 (at least 128: the tensor-core product wants that many columns); cnt[k] = padded count (0: none).
+// One CTA per clipping strength: its candidate columns in ascending order; cnt[k] = their number.
 __global__ void __launch_bounds__(1024) owc_compact_kernel(const unsigned char* __restrict__ mask, long long d_out,
                                                            int* __restrict__ idx, int* __restrict__ cnt) {
   __shared__ int s_scan[1024];
@@ -186,16 +186,30 @@ __global__ void __launch_bounds__(1024) owc_compact_kernel(const unsigned char* 
     if (tid == 0) s_base += s_scan[1023];
     __syncthreads();
   }
-  const int n = s_base;
-  const int padded = n == 0 ? 0 : (n + 127) / 128 * 128;
-  for (int t = n + tid; t < padded; t += 1024) out[t] = out[n - 1];
-  if (tid == 0) cnt[k] = padded;
+  if (tid == 0) cnt[k] = s_base;
 }
 
-__global__ void owc_scatter_kernel(const double* __restrict__ loss_c, const int* __restrict__ idx, int n,
-                                   double* __restrict__ table_row) {
+// The candidates of all strengths as one list of (column, strength) in the order of the strengths, so that the
+// exact losses take a few wide products instead of one narrow product per strength.  off[k]: where strength k's
+// candidates start (off[n_clip] = their total); entries from the total up to `padded` (a multiple of 128, the
+// granularity of the tensor-core product) repeat the last candidate.
+struct OwcOffsets { int off[257]; };
+__global__ void owc_concat_kernel(const int* __restrict__ idx, long long d_out, OwcOffsets offs, int n_clip, int padded,
+                                  int* __restrict__ cj, int* __restrict__ ck) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c < n) table_row[idx[c]] = loss_c[c];   // padding repeats a column with its own value
+  if (c >= padded) return;
+  const int total = offs.off[n_clip];
+  const int cc = c < total ? c : total - 1;
+  int k = 0;
+  while (k + 1 < n_clip && offs.off[k + 1] <= cc) ++k;
+  cj[c] = idx[(long long)k * (d_out + 128) + (cc - offs.off[k])];
+  ck[c] = k;
+}
+
+__global__ void owc_scatter_kernel(const double* __restrict__ loss_c, const int* __restrict__ cj, const int* __restrict__ ck,
+                                   int n, long long d_out, double* __restrict__ table) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < n) table[(long long)ck[c] * d_out + cj[c]] = loss_c[c];   // padding repeats a candidate with its own value
 }
 
 __global__ void fill_gamma_kernel(float* gamma_out, long long d_out) {
@@ -218,7 +232,7 @@ cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* 
 //   OWC only : gammas [n_clip] f64, gam_col [d_out] f64, table [n_clip, d_out] f64,
 //              E [d_in, d_out] f64, loss partials (FAST) or the product H E (VERIFY)
 struct InitWs {
-  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, screen, mask, idx, cnt, loss_c, total;
+  size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, screen, mask, idx, cnt, loss_c, cj, ck, total;
   bool screened;    // cheap losses first, exact ones for the near-tied strengths only
   bool tc;          // losses on the int8 tensor cores
   long long ldc;
@@ -252,6 +266,8 @@ static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n
         w.idx = take(sizeof(int) * (size_t)n_clip * (d_out + 128));
         w.cnt = take(sizeof(int) * n_clip);
         w.loss_c = take(sizeof(double) * (d_out + 128));
+        w.cj = take(sizeof(int) * ((size_t)n_clip * d_out + 128));
+        w.ck = take(sizeof(int) * ((size_t)n_clip * d_out + 128));
       }
     }
   }
@@ -321,19 +337,27 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
       if (e != cudaSuccess) return e;
       e = cudaStreamSynchronize(st);   // the sizes of the exact products are decided on the host
       if (e != cudaSuccess) return e;
-      for (int k = 0; k < n_clip; ++k) {
-        if (hcnt[k] <= 0) continue;
-        const int* idx_k = idx + (long long)k * (d_out + 128);
+      OwcOffsets offs{};
+      for (int k = 0; k < n_clip; ++k) offs.off[k + 1] = offs.off[k] + hcnt[k];
+      const int total = offs.off[n_clip], padded = (total + 127) / 128 * 128;
+      if (total <= 0) return cudaErrorUnknown;   // every column has at least its best strength as a candidate
+      int* cj = (int*)(base + L.cj);
+      int* ck = (int*)(base + L.ck);
+      { owc_concat_kernel<<<(unsigned)((padded + 255) / 256), 256, 0, st>>>(idx, d_out, offs, n_clip, padded, cj, ck); count_launch(); }
+      const int cap = (int)((d_out + 127) / 128 * 128);   // columns per product: what E, C and the slice buffers hold
+      for (int b0 = 0; b0 < padded; b0 += cap) {
+        const int width = padded - b0 < cap ? padded - b0 : cap;
         ResidualSrc src{};
         src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
-        src.mn = mn; src.mx = mx; src.gamma = hg[k]; src.L = ly.L; src.use_gamma = 1;
-        src.g = g; src.d_out = d_out; src.col_idx = idx_k; src.n_cols = hcnt[k];
+        src.mn = mn; src.mx = mx; src.L = ly.L; src.use_gamma = 1;
+        src.g = g; src.d_out = d_out; src.col_idx = cj + b0; src.n_cols = width;
+        src.col_gamma = ck + b0; src.gammas = gammas;
         e = launch_residual_f64(src, d_in, E, st);
         if (e != cudaSuccess) return e;
-        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, hcnt[k], kTcLossNE, kTcLossSmax, 1.0, (double*)(base + L.C), L.ldc,
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, width, kTcLossNE, kTcLossSmax, 1.0, (double*)(base + L.C), L.ldc,
                         loss_c, base + L.ebuf, st);
         if (e != cudaSuccess) return e;
-        { owc_scatter_kernel<<<(unsigned)((hcnt[k] + 255) / 256), 256, 0, st>>>(loss_c, idx_k, hcnt[k], table + (long long)k * d_out); count_launch(); }
+        { owc_scatter_kernel<<<(unsigned)((width + 255) / 256), 256, 0, st>>>(loss_c, cj + b0, ck + b0, width, d_out, table); count_launch(); }
       }
     } else
     for (int k = 0; k < n_clip; ++k) {
