@@ -144,9 +144,9 @@ cdq_status cdq_hessian_add_lambda(float* H, long long d_in, float lambda_rel, vo
  *   Q          [d_in, d_out] u8 out.
  *   gamma_out  [d_out] fp32 out, chosen clipping strength; may be NULL.
  * FAST, layers of at least 256 x 128: the column losses are products on the int8 tensor cores.  All
- * strengths are first screened with six slice-pair products; a strength within 2e-4 of a column's smallest
- * screened loss stays a candidate and gets the thirteen-pair loss (~1e-8 relative); the argmin is taken over
- * the candidates.  The candidate counts go through the host: one synchronisation of `stream`.
+ * strengths are first screened with three slice-pair products (six on grids of more than 4 bits); a strength
+ * within 1 % of a column's smallest screened loss stays a candidate and gets the thirteen-pair loss (~1e-8
+ * relative); the argmin is taken over the candidates.  The candidate counts go through the host: one synchronisation of `stream`.
  * The rounding decision is taken in fp64 in both modes.
  */
 cdq_status cdq_init_rtn(const void* W, cdq_dtype wt, long long d_in, long long d_out, long long ldw,

@@ -136,15 +136,18 @@ __global__ void owc_argmin_kernel(const double* __restrict__ table, int n_clip, 
 }
 
 // ---- screening of the clipping search (production mode, tensor-core losses) ----
-// The losses of all clipping strengths are first formed cheaply (six slice-pair products instead of thirteen);
+// The losses of all clipping strengths are first formed cheaply (three slice-pair products instead of thirteen);
 // a strength stays a candidate of a column if its screened loss is within kScreenBand of the column's smallest.
 // Only candidates get the thirteen-pair loss, and the argmin is taken over those: the same result as the full
-// table as long as the screening error stays inside the band.  The screen keeps three 7-bit slices of the
-// residual: the slicing truncates, and a clipped weight leaves a residual many times the typical one, so with
-// two slices (2^-14 of the column's largest residual) the screened loss was off by up to 6e-4 and picked another
-// strength on a C4-shaped layer; with three slices the error is below ~1e-5 and the band leaves a factor of 20.
-constexpr double kScreenBand = 2e-4;
-constexpr int kScreenNE = 3, kScreenSmax = 4;   // pairs (1,1) (1,2) (2,1) (1,3) (2,2) (3,1)
+// table as long as the screening error stays inside the band.  The loss as a function of the strength is smooth
+// with one minimum, and the second-best strength of a column is typically percents away (median 2.5 % on 2-bit,
+// 5 % on 3-bit grouped layers), so a band of 1 % keeps 1.1 to 1.3 candidates per column.  The screen keeps two
+// 7-bit slices of the residual and of H on grids of up to 4 bits: the slicing truncates below 2^-14 of the column's
+// largest residual, and a clipped weight leaves a residual up to (1 - gamma) L times the typical rounding error
+// (7.5 times at 4 bits), which put the screened loss off by up to 6e-4 on a 3-bit layer -- a factor of 8 inside half
+// the band.  Finer grids (L up to 255) keep three slices and six products.
+constexpr double kScreenBand = 1e-2;
+__host__ __device__ constexpr int screen_slices(int bits) { return bits <= 4 ? 2 : 3; }   // pairs up to i + j = slices + 1
 
 // mask[k][j] = 1 for candidates; the table starts at +inf everywhere.
 __global__ void owc_candidates_kernel(const double* __restrict__ screen, int n_clip, long long d_out,
@@ -326,7 +329,8 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
         src.g = g; src.d_out = d_out;
         e = launch_residual_f64(src, d_in, E, st);
         if (e != cudaSuccess) return e;
-        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, d_out, kScreenNE, kScreenSmax, 1.0, (double*)(base + L.C), L.ldc,
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, d_out, screen_slices(ly.bits), screen_slices(ly.bits) + 1, 1.0,
+                        (double*)(base + L.C), L.ldc,
                         screen + (long long)k * d_out, base + L.ebuf, st);
         if (e != cudaSuccess) return e;
       }
