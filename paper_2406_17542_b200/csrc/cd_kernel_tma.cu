@@ -268,6 +268,16 @@ cudaError_t launch_cfg(CdParams p, int nt, cudaStream_t st) {
   const size_t smem = (size_t)NCH * nt * (ROW16 ? 8 : 16) + (size_t)NCH * nt * 32 +
                       (SMODE == kPerChannel ? 0 : sizeof(float2) * (size_t)p.ag_count);
   cudaError_t e;
+  {   // rows, tables and a long list of group scales together can exceed what a block may have (18432 entries in
+      // groups of 16, say): the caller then takes the kernel that reads its rows and tables through the caches
+    cudaFuncAttributes fa{};
+    int optin = 0;
+    e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    if (smem + fa.sharedSizeBytes > (size_t)optin) return cudaErrorNotSupported;
+  }
   if (smem > 32 * 1024) {   // the 48 KB that need no opt-in include the kernel's static shared memory
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

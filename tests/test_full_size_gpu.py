@@ -182,3 +182,21 @@ def test_every_team_shape_of_the_long_row_kernel(group):
         assert stats["committed"] == budget * cfg.d_out, (d_in, stats)
         compare_with_oracle(cfg, Hd.cpu().numpy(), Hd, Wd, np.arange(cfg.d_out), g, scale, zero, Q0, Q, gamma, per, budget,
                             label=f"d_in={d_in} g={group}")
+
+
+def test_longest_rows_with_small_groups_take_the_cache_served_kernel():
+    """d_in = 18432 in groups of 16: row buffer, H_ii tables and 1152 group scales do not fit in one block's shared
+    memory together, so the descent runs in the kernel that reads rows and tables through the caches; same bars."""
+    dev = "cuda:0"
+    cfg = inputs.CONFIGS["C3"].scaled(d_in=18432, d_out=6, bits=3, group_size=16, n_clip=1, clip_lo=1.0, clip_hi=1.0, seed=77)
+    Hd = _h_from_rows(cfg, 512, ridge=1e-2)
+    Wd = inputs.make_w(cfg, device=dev)
+    g = grid_of(cfg)
+    scale, zero, Q0, gamma = B.cdq_init_rtn(Wd, g)
+    Q = Q0.clone()
+    budget = 24
+    stats, loss, per = B.cdq_cd_solve_with_loss(Hd, Wd, g, scale, zero, Q, budget, per_col=True)
+    assert B.load().cdq_last_device_status() == 0
+    assert stats["committed"] == budget * cfg.d_out
+    compare_with_oracle(cfg, Hd.cpu().numpy(), Hd, Wd, np.arange(cfg.d_out), g, scale, zero, Q0, Q, gamma, per, budget,
+                        label="d_in=18432 g=16")
