@@ -318,16 +318,20 @@ cudaError_t launch_cd_tma(const CdParams& p, cudaStream_t st) {
   // (called for rows of more than 1536 entries)  Rows up to 8192 entries: several teams per SM.
   if (ch <= 1024) return launch_mode<8, 128, 4>(p, team(ch, 8), st);
   if (ch <= 2048) return launch_mode<8, 256, 2>(p, team(ch, 8), st);
-  // Longer rows: one team per SM.  Few threads with many chunks each beat many threads with few (no spills,
-  // a cheaper argmin exchange, fixed costs per thread spread over more state), and a team of 12 or 16 full
-  // warps beats a ragged one, so the shape is the smallest of 5..8 x 512 and 7..12 x 384 chunk slots that
-  // holds the row.  Cycles per move and SM, against the 4 x 896 / 6 x 768 teams used before: d_in 10240 4526
-  // (4813), 11008 4752 (5079), 14336 5484 (5903), 15360 5865 (7482), 16384 6172 (8022), 18432 6921 (8418).
-  if (ch <= 2560) return launch_mode<5, 512, 1>(p, team(ch, 5), st);
-  if (ch <= 2688) return launch_mode<7, 384, 1>(p, team(ch, 7), st);
-  if (ch <= 3072) return launch_mode<6, 512, 1>(p, team(ch, 6), st);
-  if (ch <= 3456) return launch_mode<9, 384, 1>(p, team(ch, 9), st);
-  if (ch <= 3584) return launch_mode<7, 512, 1>(p, team(ch, 7), st);
+  // Longer rows: one team per SM.  Few threads with many chunks each beat many threads with few (no spills, a
+  // cheaper argmin exchange, fixed costs per thread spread over more state), and a team of full warps in equal
+  // numbers per scheduler beats a ragged one.  With H_ii and 0.5 / H_ii in shared memory eight warps hide the
+  // latencies that are left, so rows up to 14336 entries take 256 threads with 9 to 14 chunks each; beyond that the
+  // registers of a 256-thread team run out (15 and 16 chunks measured 3 % slower, 18 chunks 15 %) and the team is the
+  // smallest of 10..12 x 384 and 8 x 512 chunk slots that holds the row.  Cycles per move and SM against the
+  // 4 x 896 / 6 x 768 teams of an earlier version, which also read the tables through L1: d_in 10240 4049 (4813),
+  // 11008 4038 (5079), 14336 4892 (5903), 15360 5531 (7482), 16384 5879 (8022), 18432 6416 (8418).
+  if (ch <= 2304) return launch_mode<9, 256, 1>(p, team(ch, 9), st);
+  if (ch <= 2560) return launch_mode<10, 256, 1>(p, team(ch, 10), st);
+  if (ch <= 2816) return launch_mode<11, 256, 1>(p, team(ch, 11), st);
+  if (ch <= 3072) return launch_mode<12, 256, 1>(p, team(ch, 12), st);
+  if (ch <= 3328) return launch_mode<13, 256, 1>(p, team(ch, 13), st);
+  if (ch <= 3584) return launch_mode<14, 256, 1>(p, team(ch, 14), st);
   if (ch <= 3840) return launch_mode<10, 384, 1>(p, team(ch, 10), st);
   if (ch <= 4096) return launch_mode<8, 512, 1>(p, team(ch, 8), st);
   if (ch <= 4224) return launch_mode<11, 384, 1>(p, team(ch, 11), st);

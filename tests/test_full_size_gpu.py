@@ -156,7 +156,7 @@ def test_long_columns_whose_length_is_not_a_multiple_of_four_sampled():
 # Row lengths (in entries) at which the kernel that stages rows through shared memory changes its team shape,
 # each with a length just inside the next shape; 12224 and 12288 are the lengths whose row fills the 48 KB of
 # shared memory that need no opt-in (together with the kernel's own static shared memory they exceed it).
-_SHAPE_EDGES = [4 * c for c in (1024, 2048, 2560, 2688, 3072, 3456, 3584, 3840, 4096, 4224, 4608)]
+_SHAPE_EDGES = [4 * c for c in (1024, 2048, 2304, 2560, 2816, 3072, 3328, 3584, 3840, 4096, 4224, 4608)]
 ROW_LENGTHS = {
     0: sorted(set([2304, 12224] + _SHAPE_EDGES + [d + 16 for d in _SHAPE_EDGES[:-1]])),
     128: sorted(set([2304, 12160] + _SHAPE_EDGES + [d + 128 for d in _SHAPE_EDGES[:-1]])),
