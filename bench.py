@@ -43,7 +43,7 @@ L2_BYTES = 126e6
 # capture divided by the moves of that capture), keyed by (kernel, d_in); a kernel and shape without a
 # capture of the kernel as it stands reports traffic null.  Each entry names the summary it comes from.
 NCU_TRAFFIC_PER_MOVE: dict = {
-    ("cd_tma_kernel", 14336): (44542.0, "profiles/cd_tma_kernel_C3_592cols.md"),
+    ("cd_tma_kernel", 14336): (44533.0, "profiles/cd_tma_kernel_C3_592cols.md"),
 }
 
 
