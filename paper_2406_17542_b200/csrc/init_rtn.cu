@@ -209,6 +209,15 @@ __global__ void owc_concat_kernel(const int* __restrict__ idx, long long d_out, 
   ck[c] = k;
 }
 
+// Columns of a screening product over several strengths at once: column c is layer column c % d_out under strength
+// k0 + c / d_out.
+__global__ void owc_iota_kernel(long long d_out, int k0, long long width, int* __restrict__ cj, int* __restrict__ ck) {
+  const long long c = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (c >= width) return;
+  cj[c] = (int)(c % d_out);
+  ck[c] = k0 + (int)(c / d_out);
+}
+
 __global__ void owc_scatter_kernel(const double* __restrict__ loss_c, const int* __restrict__ cj, const int* __restrict__ ck,
                                    int n, long long d_out, double* __restrict__ table) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -237,6 +246,8 @@ cudaError_t launch_group_minmax(const Layer& ly, float* pmn, float* pmx, float* 
 struct InitWs {
   size_t pmn, pmx, mn, mx, gammas, gam_col, table, E, part, C, hbuf, ebuf, screen, mask, idx, cnt, loss_c, cj, ck, total;
   bool screened;    // cheap losses first, exact ones for the near-tied strengths only
+  int sbatch;       // strengths per screening product (several on small layers, where a product per strength is launch-bound)
+  long long wcap;   // columns that E, C and the slice buffers hold
   bool tc;          // losses on the int8 tensor cores
   long long ldc;
 };
@@ -254,21 +265,27 @@ static InitWs init_ws_layout(long long d_in, long long d_out, long long g, int n
     w.gammas = take(sizeof(double) * n_clip);
     w.gam_col = take(sizeof(double) * d_out);
     w.table = take(sizeof(double) * n_clip * d_out);
-    w.E = take(sizeof(double) * d_in * (d_out + 128));
-    w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
     w.tc = mode == CDQ_MODE_FAST && gemm_tc_supported(d_in, d_out);
+    w.screened = w.tc && n_clip >= 4;
+    w.sbatch = 1;
+    if (w.screened) {   // up to 1 GiB of residuals per product
+      const long long fit = (1ll << 30) / (8 * d_in * d_out);
+      w.sbatch = (int)(fit < 1 ? 1 : (fit > n_clip ? n_clip : fit));
+    }
+    w.wcap = d_out + 128 > (long long)w.sbatch * d_out ? d_out + 128 : (long long)w.sbatch * d_out;
+    w.E = take(sizeof(double) * d_in * w.wcap);
+    w.part = take(sizeof(double) * (mode == CDQ_MODE_FAST ? gemm_partials_elems(d_in, d_out) : (size_t)d_in * d_out));
     w.ldc = (d_in + 3) / 4 * 4;
     if (w.tc) {
-      w.C = take(sizeof(double) * (d_out + 128) * w.ldc);
+      w.C = take(sizeof(double) * w.wcap * w.ldc);
       w.hbuf = take(gemm_tc_h_bytes(d_in, kTcLossNH));
-      w.ebuf = take(gemm_tc_e_bytes(d_in, d_out + 128, kTcLossNE));
-      w.screened = n_clip >= 4;
+      w.ebuf = take(gemm_tc_e_bytes(d_in, w.wcap, kTcLossNE));
       if (w.screened) {
         w.screen = take(sizeof(double) * n_clip * d_out);
         w.mask = take((size_t)n_clip * d_out);
         w.idx = take(sizeof(int) * (size_t)n_clip * (d_out + 128));
         w.cnt = take(sizeof(int) * n_clip);
-        w.loss_c = take(sizeof(double) * (d_out + 128));
+        w.loss_c = take(sizeof(double) * w.wcap);
         w.cj = take(sizeof(int) * ((size_t)n_clip * d_out + 128));
         w.ck = take(sizeof(int) * ((size_t)n_clip * d_out + 128));
       }
@@ -322,16 +339,23 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
       int* idx = (int*)(base + L.idx);
       int* cnt = (int*)(base + L.cnt);
       double* loss_c = (double*)(base + L.loss_c);
-      for (int k = 0; k < n_clip; ++k) {   // screening
+      int* cj = (int*)(base + L.cj);
+      int* ck = (int*)(base + L.ck);
+      for (int k0 = 0; k0 < n_clip; k0 += L.sbatch) {   // screening, L.sbatch strengths per product
+        const int gb = n_clip - k0 < L.sbatch ? n_clip - k0 : L.sbatch;
+        const long long width = (long long)gb * d_out;
         ResidualSrc src{};
         src.W = ly.W; src.wt = ly.wt; src.ldw = ly.ldw;
-        src.mn = mn; src.mx = mx; src.gamma = hg[k]; src.L = ly.L; src.use_gamma = 1;
+        src.mn = mn; src.mx = mx; src.gamma = hg[k0]; src.L = ly.L; src.use_gamma = 1;
         src.g = g; src.d_out = d_out;
+        if (gb > 1) {
+          { owc_iota_kernel<<<(unsigned)((width + 255) / 256), 256, 0, st>>>(d_out, k0, width, cj, ck); count_launch(); }
+          src.col_idx = cj; src.n_cols = width; src.col_gamma = ck; src.gammas = gammas;
+        }
         e = launch_residual_f64(src, d_in, E, st);
         if (e != cudaSuccess) return e;
-        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, d_out, screen_slices(ly.bits), screen_slices(ly.bits) + 1, 1.0,
-                        (double*)(base + L.C), L.ldc,
-                        screen + (long long)k * d_out, base + L.ebuf, st);
+        e = gemm_tc_run(base + L.hbuf, kTcLossNH, E, d_in, width, screen_slices(ly.bits), screen_slices(ly.bits) + 1, 1.0,
+                        (double*)(base + L.C), L.ldc, screen + (long long)k0 * d_out, base + L.ebuf, st);
         if (e != cudaSuccess) return e;
       }
       { owc_candidates_kernel<<<bx, 128, 0, st>>>(screen, n_clip, d_out, mask, table); count_launch(); }
@@ -345,10 +369,8 @@ cudaError_t launch_init_rtn(const Layer& ly, const cdq_grid_desc& grid, float* s
       for (int k = 0; k < n_clip; ++k) offs.off[k + 1] = offs.off[k] + hcnt[k];
       const int total = offs.off[n_clip], padded = (total + 127) / 128 * 128;
       if (total <= 0) return cudaErrorUnknown;   // every column has at least its best strength as a candidate
-      int* cj = (int*)(base + L.cj);
-      int* ck = (int*)(base + L.ck);
       { owc_concat_kernel<<<(unsigned)((padded + 255) / 256), 256, 0, st>>>(idx, d_out, offs, n_clip, padded, cj, ck); count_launch(); }
-      const int cap = (int)((d_out + 127) / 128 * 128);   // columns per product: what E, C and the slice buffers hold
+      const int cap = (int)(L.wcap / 128 * 128);   // columns per product: what E, C and the slice buffers hold
       for (int b0 = 0; b0 < padded; b0 += cap) {
         const int width = padded - b0 < cap ? padded - b0 : cap;
         ResidualSrc src{};
