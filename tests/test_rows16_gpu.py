@@ -32,8 +32,8 @@ def _h_from_rows(cfg, rows, ridge=1e-3):
     ("C3", 4608, 64, 0, 4, 4096, 64),          # two 256-thread teams per SM
     ("C3", 6144, 148, 0, 3, 4096, 32),
     ("C3", 11008, 148, 0, 4, 4096, 16),        # ragged: the last chunk slots reach past the row
-    ("C3", 14336, 296, 0, 4, 8192, 24),        # the C3 team (896 x 4), whole row in one copy
-    ("C4", 18432, 148, 128, 3, 4096, 12),      # the C4 team (768 x 6), groups of 128, one copy per chunk slot
+    ("C3", 14336, 296, 0, 4, 8192, 24),        # the C3 team (256 threads x 14 chunks)
+    ("C4", 18432, 148, 128, 3, 4096, 12),      # the C4 team (384 threads x 12 chunks), groups of 128
 ])
 def test_bf16_rows_against_the_oracle_on_the_rounded_matrix(name, d_in, d_out, g, bits, rows, n_sample):
     cfg = inputs.CONFIGS[name].scaled(d_in=d_in, d_out=d_out, group_size=g, bits=bits, n_clip=1, clip_lo=1.0, clip_hi=1.0,
